@@ -1,0 +1,220 @@
+/*
+ * fc.h — C ABI of the FlowCache hot path for NVIDIA B200 (sm_100a).
+ *
+ * FlowCache (arXiv 2602.10825) is a chunkwise caching scheme for autoregressive
+ * video diffusion transformers.  This library implements the per-denoising-step
+ * chunk pipeline as four calls, all enqueued on a caller-supplied CUDA stream:
+ *
+ *   fc_chunk_decide       which chunks are recomputed at this step   (Eqs. 5, 8)
+ *   fc_chunk_attention    attention of the recomputed chunks' queries over the
+ *                         fixed-budget KV cache plus the denoising window (Sec. 3.3)
+ *   fc_kv_score           importance / redundancy score of cached tokens (Eqs. 9-12)
+ *   fc_kv_select_compact  per-head top-B and retention of the chosen K/V rows
+ *
+ * Conventions
+ *   - Plain C types only.  Every pointer argument says whether it is a HOST or a
+ *     DEVICE pointer.  The caller owns every buffer, including the workspace,
+ *     whose size the matching fc_*_workspace_bytes() returns.  No call allocates
+ *     or frees device memory, synchronises the host with the device, or uses a
+ *     stream other than `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream).
+ *   - Tensors are [heads, tokens, d] with d contiguous and explicit head / token
+ *     strides counted in elements.  Device base pointers must be 16-byte aligned
+ *     and every stride a multiple of 16 bytes.
+ *   - dtype is the storage type of the tensors (FC_BF16 or FC_F32); sums and
+ *     softmax statistics are always kept in fp32 or wider.
+ *   - Return value: FC_OK (0) or a negative fc_status.  On an error nothing has
+ *     been launched.  Data-dependent conditions that can only be seen on the
+ *     device (a NaN score, a bounded wait that expired) set bits in the optional
+ *     DEVICE word `status` (OR-ed in, never cleared by the library); the caller
+ *     reads it after its own synchronisation.
+ *   - The library keeps no state between calls except immutable per-device
+ *     attributes inside fc_ctx.  Calls on different streams may overlap as long
+ *     as their buffers and workspaces do not.
+ */
+#ifndef FC_H_
+#define FC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FC_OK = 0,
+  FC_ERR_INVALID_ARG = -1, /* NULL where a pointer is required, negative size, even pool_k ... */
+  FC_ERR_UNSUPPORTED = -2, /* d not in {64,128}, unknown dtype, too many chunks / segments */
+  FC_ERR_MISALIGNED = -3,  /* a base pointer or stride is not a multiple of 16 bytes */
+  FC_ERR_WORKSPACE = -4,   /* ws is NULL or ws_bytes is below fc_*_workspace_bytes() */
+  FC_ERR_DEVICE = -5,      /* the device is not compute capability 10.x */
+  FC_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed (see fc_last_cuda_error) */
+  FC_ERR_UNIMPLEMENTED = -7
+} fc_status;
+
+typedef enum { FC_BF16 = 0, FC_F32 = 1 } fc_dtype;
+
+/* Bits of the device status word. */
+enum {
+  FC_DEV_TIMEOUT = 1u,   /* a bounded in-kernel wait expired; the affected outputs are invalid */
+  FC_DEV_NAN_SCORE = 2u, /* a NaN score was ranked as -inf by the selection */
+  FC_DEV_BAD_INDEX = 4u  /* an index read from device memory was out of range and was skipped */
+};
+
+enum { FC_MAX_CHUNKS = 64, FC_MAX_SEGMENTS = 64 };
+
+typedef struct fc_ctx fc_ctx;
+
+/* Create / destroy a context for CUDA device `device` (made current by the call).  Reads the
+ * device attributes (SM count, shared-memory limit) and resolves the driver entry point used to
+ * encode TMA tensor maps.  Fails with FC_ERR_DEVICE unless the device is compute capability 10.x. */
+int fc_create(fc_ctx** out, int device);
+int fc_destroy(fc_ctx* ctx);
+const char* fc_status_string(int status);
+/* Text of the last CUDA error a call on this thread ran into ("" if none). */
+const char* fc_last_cuda_error(void);
+/* Number of SMs the context's persistent kernels size their grids by. */
+int fc_sm_count(const fc_ctx* ctx);
+
+/* ------------------------------------------------------------------------------------------
+ * fc_chunk_decide — per-chunk reuse decision.
+ *
+ * Paper: the relative L1 distance of chunk i between consecutive denoising steps (Eq. 5, the
+ * per-chunk form of Eq. 4) is accumulated per chunk and compared with a threshold (Eq. 8):
+ *     r_i = sum|cur_i - prev_i| / sum|prev_i|           (the denominator is the earlier state)
+ *     s_i = acc_i + r_i                                 (fp32)
+ *     recompute_i = chunk_step[i] < warmup_m  ||  force[i]  ||  s_i > eps      (strict)
+ *     acc_i <- 0 if recompute_i else s_i
+ * A zero denominator yields r = +inf if the numerator is positive, else 0.
+ *
+ *   cur, prev        DEVICE, `dtype` elements; chunk i occupies elements
+ *                    [chunk_elem_off[i], chunk_elem_off[i+1]) of both.  The vectorised path
+ *                    is taken when every offset is a multiple of 16 bytes.
+ *   chunk_elem_off   HOST [n_chunks+1], non-decreasing; n_chunks <= FC_MAX_CHUNKS.
+ *   chunk_step       DEVICE [n_chunks]: number of steps chunk i has already taken.
+ *   force            DEVICE [n_chunks] or NULL: non-zero forces a recompute (a newly
+ *                    initialised chunk must be computed).
+ *   acc              DEVICE [n_chunks], in/out: the accumulator f of Eq. 8.
+ *   l1rel            DEVICE [n_chunks] out or NULL: r_i.
+ *   recompute        DEVICE [n_chunks] out: 1 = recompute, 0 = serve from cache.
+ *   active_ids       DEVICE [n_chunks] out: ids of recomputed chunks, ascending; entries at
+ *                    and after n_active are set to -1.
+ *   n_active         DEVICE [1] out.
+ * Sums are fixed-order (run-to-run bit-reproducible): fp32 inside a thread's 32-element run,
+ * fp64 above that.  Workspace: fc_chunk_decide_workspace_bytes(total elements, n_chunks). */
+size_t fc_chunk_decide_workspace_bytes(int64_t total_elems, int n_chunks);
+int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
+                    const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
+                    int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
+                    uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
+                    uint32_t* status, void* ws, size_t ws_bytes);
+
+/* ------------------------------------------------------------------------------------------
+ * fc_chunk_attention — chunk-causal attention of the active chunks.
+ *
+ * Paper (Sec. 3.3): the chunks being denoised attend to the compressed clean-chunk region of
+ * the KV buffer followed by the current denoising region; generation is causal over chunks.
+ * For every active chunk c, head h and query row r of c:
+ *     O[h, r, :] = softmax_j( Q[h, r, :] . K[g(h), p(j), :] * scale ) V[g(h), p(j), :],
+ *     j over the first kv_visible_len[c] LOGICAL tokens, g(h) = h / (H_q / H_kv),
+ * where p maps a logical token to a physical row of the K/V store: through the segment table
+ * (logical range [seg_logical_off[s], seg_logical_off[s+1]) starts at physical row
+ * seg_phys_off[s]) or, if given, through the per-head token map kv_token_index[g][j] (this is
+ * how a cache is read through the kept-index list of fc_kv_select_compact without moving it).
+ * All tokens of a chunk's own range are visible to all its rows (no mask inside a chunk).
+ * Rows of chunks that are not in active_ids are never written: their cached outputs stay.
+ */
+typedef struct {
+  int32_t H_q, H_kv, d, W;                   /* query heads, kv heads, head dim (64|128), chunks */
+  int64_t q_hs, q_rs, k_hs, k_rs, v_hs, v_rs; /* element strides: head, row */
+  int64_t o_hs, o_rs;
+  int64_t kv_rows;                           /* physical rows per head in the K/V store */
+  float scale;                               /* 0 => 1/sqrt(d) */
+  int32_t impl;                              /* 0 auto; 1 force the CUDA-core kernel; 2 force tcgen05 */
+} fc_attn_desc;
+
+/*   Q, O             DEVICE [H_q, rows, d]; K, V DEVICE [H_kv, kv_rows, d]; `dtype` elements.
+ *   q_chunk_row_off  HOST [W+1]: chunk c owns query rows [off[c], off[c+1]).  W <= FC_MAX_CHUNKS.
+ *   kv_visible_len   HOST [W].
+ *   seg_logical_off  HOST [n_seg+1], seg_phys_off HOST [n_seg]; n_seg <= FC_MAX_SEGMENTS.
+ *                    Ignored (may be NULL, n_seg 0) when kv_token_index is given.
+ *   kv_token_index   DEVICE [H_kv, kv_index_hs] int32 or NULL.
+ *   active_ids       DEVICE [<= W], n_active DEVICE [1] (as written by fc_chunk_decide): the
+ *                    work list is read on the device, so no host synchronisation is needed
+ *                    between the decision and the attention.
+ *   lse              DEVICE [H_q, lse_hs] fp32 or NULL: natural-log sum-exp of each computed row.
+ * bf16 runs on tcgen05 tensor cores (fp32 accumulation in tensor memory, TMA-fed); fp32 runs
+ * on CUDA cores with fp32 accumulation.  Workspace: fc_chunk_attention_workspace_bytes(). */
+size_t fc_chunk_attention_workspace_bytes(const fc_attn_desc* desc);
+int fc_chunk_attention(fc_ctx* ctx, void* stream, const fc_attn_desc* desc, const void* Q,
+                       const void* K, const void* V, int dtype, const int32_t* q_chunk_row_off,
+                       const int32_t* kv_visible_len, const int32_t* seg_logical_off,
+                       const int32_t* seg_phys_off, int n_seg, const int32_t* kv_token_index,
+                       int64_t kv_index_hs, const int32_t* active_ids, const int32_t* n_active,
+                       void* O, float* lse, int64_t lse_hs, uint32_t* status, void* ws,
+                       size_t ws_bytes);
+
+/* ------------------------------------------------------------------------------------------
+ * fc_kv_score — joint importance / redundancy score of the candidate tokens.
+ *
+ * Paper: Imp_j = mean over the observation queries (and the query heads of a kv head's group)
+ * of softmax_j(q K_cand^T * scale) (Eq. 9); Imp~ = stride-1 max-pool of width pool_k with
+ * -inf padding (Eq. 10); Red_j = softmax_j of the column means of the cosine-similarity matrix
+ * of the l2-normalised keys with a zeroed diagonal (Eq. 11), evaluated through the mean-key
+ * identity of the paper's efficiency appendix, column mean_j = (mean_i khat_i).khat_j -
+ * |khat_j|^2 / L_k, with khat = k / max(|k|, 1e-12); Score = lambda*Imp~ - (1-lambda)*Red (Eq. 12).
+ */
+typedef struct {
+  int32_t H_q, H_kv, d, L_q, L_k;  /* L_q * (H_q/H_kv) <= 128 */
+  int64_t q_hs, q_rs, k_hs, k_rs;  /* element strides */
+  float scale;                     /* 0 => 1/sqrt(d) */
+  float lambda;                    /* mixing coefficient (paper: 0.07) */
+  int32_t pool_k;                  /* odd, >= 1 */
+  int32_t impl;                    /* 0 auto; 1 force the CUDA-core kernels; 2 force tcgen05 */
+} fc_score_desc;
+
+/*   Q_obs            DEVICE [H_q, L_q, d]; K_cand DEVICE [H_kv, L_k, d]; `dtype` elements.
+ *   imp_accum        DEVICE [H_kv, L_k] fp32 or NULL; accum_phase: 0 single shot (imp_accum
+ *                    unused); 1 imp_accum += Imp of this call, nothing else is written; 2
+ *                    imp_accum += Imp, then Imp := imp_accum / n_steps and the scores are
+ *                    finalised (mean importance over the steps of a chunk).
+ *   imp, red         DEVICE [H_kv, L_k] fp32 out, either may be NULL.
+ *   score            DEVICE [H_kv, L_k] fp32 out (required unless accum_phase == 1).
+ * Deterministic: no floating-point atomics.  Workspace: fc_kv_score_workspace_bytes(). */
+size_t fc_kv_score_workspace_bytes(const fc_score_desc* desc);
+int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc, const void* Q_obs,
+                const void* K_cand, int dtype, float* imp_accum, int accum_phase, int n_steps,
+                float* imp, float* red, float* score, uint32_t* status, void* ws,
+                size_t ws_bytes);
+
+/* ------------------------------------------------------------------------------------------
+ * fc_kv_select_compact — per-head top-B and retention of the selected rows.
+ *
+ * Paper: for each head keep the B tokens with the highest Score (text after Eq. 12); the kept
+ * K/V form the compressed clean region (Sec. 3.3).  Total order: score descending, index
+ * ascending (so ties keep the lowest indices); NaN ranks as -inf and sets FC_DEV_NAN_SCORE;
+ * -0 equals +0.  B >= L_k keeps everything (identity).
+ *
+ *   score            DEVICE [n_heads, L_k] fp32.
+ *   K_src, V_src     DEVICE [n_heads, L_k, d] with strides src_hs / src_rs (elements);
+ *   K_dst, V_dst     DEVICE [n_heads, >= min(B,L_k), d] with strides dst_hs / dst_rs; must not
+ *                    overlap the sources.  All four NULL => selection only.
+ *   kept_idx         DEVICE [n_heads, min(B, L_k)] int32 out, ascending per head.
+ *   n_kept           DEVICE [1] out or NULL: min(B, L_k).
+ * Row r of head h of the destination is source row kept_idx[h][r], copied byte for byte with
+ * 16-byte accesses; bytes outside the kept rows are not touched; dropped rows are not read. */
+typedef struct {
+  int64_t src_hs, src_rs, dst_hs, dst_rs;
+} fc_compact_strides;
+
+size_t fc_kv_select_compact_workspace_bytes(int n_heads, int L_k);
+int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* score, int n_heads, int L_k,
+                         int B, const void* K_src, const void* V_src, void* K_dst, void* V_dst,
+                         int dtype, int d, const fc_compact_strides* strides, int32_t* kept_idx,
+                         int32_t* n_kept, uint32_t* status, void* ws, size_t ws_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FC_H_ */

@@ -1,0 +1,31 @@
+// Geometry shared by the two attention kernels of libfc (CUDA-core and tcgen05).
+#pragma once
+
+#include "fc_common.cuh"
+
+namespace fc {
+
+struct AttnGeom {
+  int32_t H_q, H_kv, d, W, group, n_seg;
+  int64_t q_hs, q_rs, k_hs, k_rs, v_hs, v_rs, o_hs, o_rs, kv_rows, lse_hs, tok_hs;
+  float scale;
+  int32_t q_row_off[FC_MAX_CHUNKS + 1];
+  int32_t vis[FC_MAX_CHUNKS];
+  int32_t seg_log[FC_MAX_SEGMENTS + 1];
+  int32_t seg_phys[FC_MAX_SEGMENTS];
+  const int32_t* tok_index;
+  const int32_t* active_ids;
+  const int32_t* n_active;
+  float* lse;
+  uint32_t* status;
+};
+
+int attention_simt(cudaStream_t st, const AttnGeom& g, const void* Q, const void* K, const void* V,
+                   int dtype, void* O);
+// bf16 only, segment-table addressing only.
+int attention_tc(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const void* Q, const void* K,
+                 const void* V, void* O, void* ws, size_t ws_bytes);
+size_t attention_tc_workspace_bytes();
+bool attention_tc_supported(const AttnGeom& g, int dtype);
+
+}  // namespace fc

@@ -1,0 +1,67 @@
+// Internal helpers shared by the kernels of libfc (never by the CPU oracle).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fc.h"
+
+struct fc_ctx {
+  int device;
+  int sm_count;
+  int smem_optin;       // max dynamic shared memory per block (opt-in), bytes
+  void* encode_tiled;   // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+namespace fc {
+
+void set_cuda_error(cudaError_t e, const char* where);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int elem_size(int dtype) { return dtype == FC_F32 ? 4 : 2; }
+
+#define FC_CUDA_CHECK(expr)                         \
+  do {                                              \
+    cudaError_t e__ = (expr);                       \
+    if (e__ != cudaSuccess) {                       \
+      fc::set_cuda_error(e__, #expr);               \
+      return FC_ERR_CUDA;                           \
+    }                                               \
+  } while (0)
+
+#define FC_LAUNCH_CHECK(name)                       \
+  do {                                              \
+    cudaError_t e__ = cudaGetLastError();           \
+    if (e__ != cudaSuccess) {                       \
+      fc::set_cuda_error(e__, name);                \
+      return FC_ERR_CUDA;                           \
+    }                                               \
+  } while (0)
+
+// Storage element -> float.
+template <typename T> __device__ __forceinline__ float to_float(T x);
+template <> __device__ __forceinline__ float to_float<float>(float x) { return x; }
+template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 x) {
+  return __bfloat162float(x);
+}
+
+// Two bf16 packed in a 32-bit word -> two floats (exact: bf16 is the top half of an fp32).
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream16(void* p, uint4 v) {
+  asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+               "r"(v.w)
+               : "memory");
+}
+
+}  // namespace fc

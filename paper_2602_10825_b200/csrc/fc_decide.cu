@@ -1,0 +1,211 @@
+// fc_chunk_decide: per-chunk relative-L1 indicator (Eq. 5) and the accumulate / threshold /
+// reset rule (Eq. 8).
+//
+// Two launches.  (1) A streaming segmented reduction: the chunks are cut into slabs of 16 KiB
+// per tensor, one block per slab; every thread sums |cur-prev| and |prev| of 4 interleaved
+// 16-byte vectors in fp32, the block combines them in fp64 in a fixed tree and writes one
+// (num, den) pair per slab.  (2) One block: a warp per chunk adds that chunk's slab pairs in a
+// fixed order in fp64, forms r, applies the rule in fp32 and compacts the active ids.
+// No atomics: results are bit-reproducible from run to run.
+#include "fc_common.cuh"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kVecPerThread = 4;
+constexpr int kSlabBytes = kThreads * kVecPerThread * 16;  // per tensor
+
+struct DecideGeom {
+  int64_t elem_off[FC_MAX_CHUNKS + 1];
+  int32_t slab_off[FC_MAX_CHUNKS + 1];
+  int32_t n_chunks;
+};
+
+__device__ __forceinline__ void accum_vec(const uint4& c, const uint4& p, __nv_bfloat16*, float& num,
+                                          float& den) {
+  const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, pw[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float c0 = fc::bf16_lo(cw[i]), c1 = fc::bf16_hi(cw[i]);
+    float p0 = fc::bf16_lo(pw[i]), p1 = fc::bf16_hi(pw[i]);
+    num += fabsf(c0 - p0);
+    den += fabsf(p0);
+    num += fabsf(c1 - p1);
+    den += fabsf(p1);
+  }
+}
+__device__ __forceinline__ void accum_vec(const uint4& c, const uint4& p, float*, float& num, float& den) {
+  const uint32_t cw[4] = {c.x, c.y, c.z, c.w}, pw[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float cf = __uint_as_float(cw[i]), pf = __uint_as_float(pw[i]);
+    num += fabsf(cf - pf);
+    den += fabsf(pf);
+  }
+}
+
+template <typename T, bool kVec>
+__global__ void __launch_bounds__(kThreads)
+decide_partial_kernel(const T* __restrict__ cur, const T* __restrict__ prev, DecideGeom g,
+                      double2* __restrict__ partial) {
+  constexpr int kElemPerVec = 16 / (int)sizeof(T);
+  constexpr int kSlabElems = kSlabBytes / (int)sizeof(T);
+  const int b = blockIdx.x;
+  int c = 0;
+  while (c + 1 < g.n_chunks && b >= g.slab_off[c + 1]) ++c;
+  const int64_t begin = g.elem_off[c] + (int64_t)(b - g.slab_off[c]) * kSlabElems;
+  const int64_t end = min(begin + (int64_t)kSlabElems, g.elem_off[c + 1]);
+  float num = 0.f, den = 0.f;
+  if (kVec) {
+    uint4 cv[kVecPerThread], pv[kVecPerThread];
+    bool ok[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+      const int64_t e = begin + (int64_t)(k * kThreads + threadIdx.x) * kElemPerVec;
+      ok[k] = e < end;  // chunk lengths are vector multiples on this path
+      if (ok[k]) {
+        cv[k] = fc::ld_stream16(cur + e);
+        pv[k] = fc::ld_stream16(prev + e);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k)
+      if (ok[k]) accum_vec(cv[k], pv[k], (T*)nullptr, num, den);
+  } else {
+    for (int64_t e = begin + threadIdx.x; e < end; e += kThreads) {
+      float cf = fc::to_float(cur[e]), pf = fc::to_float(prev[e]);
+      num += fabsf(cf - pf);
+      den += fabsf(pf);
+    }
+  }
+  double dn = (double)num, dd = (double)den;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    dn += __shfl_down_sync(0xffffffffu, dn, o);
+    dd += __shfl_down_sync(0xffffffffu, dd, o);
+  }
+  __shared__ double2 warp_sum[kThreads / 32];
+  if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = make_double2(dn, dd);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double2 s = warp_sum[0];
+    for (int w = 1; w < kThreads / 32; ++w) {
+      s.x += warp_sum[w].x;
+      s.y += warp_sum[w].y;
+    }
+    partial[b] = s;
+  }
+}
+
+__global__ void __launch_bounds__(1024)
+decide_finalize_kernel(DecideGeom g, const double2* __restrict__ partial,
+                       const int32_t* __restrict__ chunk_step, int warmup_m, float eps,
+                       const uint8_t* __restrict__ force, float* __restrict__ acc,
+                       float* __restrict__ l1rel, uint8_t* __restrict__ recompute,
+                       int32_t* __restrict__ active_ids, int32_t* __restrict__ n_active) {
+  __shared__ uint8_t flag[FC_MAX_CHUNKS];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int c = warp; c < g.n_chunks; c += 32) {
+    double num = 0.0, den = 0.0;
+    for (int s = g.slab_off[c] + lane; s < g.slab_off[c + 1]; s += 32) {
+      num += partial[s].x;
+      den += partial[s].y;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      num += __shfl_down_sync(0xffffffffu, num, o);
+      den += __shfl_down_sync(0xffffffffu, den, o);
+    }
+    if (lane == 0) {
+      double r;
+      if (den > 0.0)
+        r = num / den;
+      else
+        r = num > 0.0 ? (double)INFINITY : 0.0;
+      const float rf = (float)r;
+      const float s = __fadd_rn(acc[c], rf);
+      const bool rec = chunk_step[c] < warmup_m || (force && force[c]) || s > eps;
+      if (l1rel) l1rel[c] = rf;
+      recompute[c] = rec ? 1 : 0;
+      acc[c] = rec ? 0.f : s;
+      flag[c] = rec ? 1 : 0;
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = 0;
+    for (int c = 0; c < g.n_chunks; ++c)
+      if (flag[c]) active_ids[n++] = c;
+    *n_active = n;
+    for (int c = n; c < g.n_chunks; ++c) active_ids[c] = -1;
+  }
+}
+
+int64_t slab_elems(int dtype) { return kSlabBytes / fc::elem_size(dtype); }
+
+}  // namespace
+
+extern "C" size_t fc_chunk_decide_workspace_bytes(int64_t total_elems, int n_chunks) {
+  if (total_elems < 0 || n_chunks < 0) return 0;
+  // one (num, den) pair per slab; slabs never straddle chunks, sized for the narrower dtype
+  const int64_t slabs = total_elems / slab_elems(FC_F32) + n_chunks + 1;
+  return (size_t)slabs * sizeof(double2);
+}
+
+extern "C" int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
+                               const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
+                               int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
+                               uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
+                               uint32_t* status, void* ws, size_t ws_bytes) {
+  (void)status;
+  if (!ctx || !chunk_elem_off || !chunk_step || !acc || !recompute || !active_ids || !n_active)
+    return FC_ERR_INVALID_ARG;
+  if (n_chunks <= 0) return FC_ERR_INVALID_ARG;
+  if (n_chunks > FC_MAX_CHUNKS) return FC_ERR_UNSUPPORTED;
+  if (dtype != FC_BF16 && dtype != FC_F32) return FC_ERR_UNSUPPORTED;
+  const int es = fc::elem_size(dtype);
+  DecideGeom g;
+  g.n_chunks = n_chunks;
+  const int64_t se = slab_elems(dtype);
+  bool vec = fc::aligned16(cur) && fc::aligned16(prev);
+  int64_t slabs = 0;
+  for (int c = 0; c <= n_chunks; ++c) {
+    g.elem_off[c] = chunk_elem_off[c];
+    if (chunk_elem_off[c] < 0 || (c > 0 && chunk_elem_off[c] < chunk_elem_off[c - 1]))
+      return FC_ERR_INVALID_ARG;
+    if ((chunk_elem_off[c] * es) % 16) vec = false;
+    g.slab_off[c] = (int32_t)slabs;
+    if (c < n_chunks) slabs += (chunk_elem_off[c + 1] - chunk_elem_off[c] + se - 1) / se;
+    if (slabs > INT32_MAX / 2) return FC_ERR_UNSUPPORTED;
+  }
+  const int64_t total = chunk_elem_off[n_chunks];
+  if (total > 0 && (!cur || !prev)) return FC_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < (size_t)slabs * sizeof(double2) ||
+      ws_bytes < fc_chunk_decide_workspace_bytes(total, n_chunks))
+    return FC_ERR_WORKSPACE;
+  if (!fc::aligned16(ws)) return FC_ERR_MISALIGNED;
+  cudaStream_t st = (cudaStream_t)stream;
+  double2* partial = (double2*)ws;
+  if (slabs > 0) {
+    if (dtype == FC_BF16) {
+      auto* c = (const __nv_bfloat16*)cur;
+      auto* p = (const __nv_bfloat16*)prev;
+      if (vec)
+        decide_partial_kernel<__nv_bfloat16, true><<<(unsigned)slabs, kThreads, 0, st>>>(c, p, g, partial);
+      else
+        decide_partial_kernel<__nv_bfloat16, false><<<(unsigned)slabs, kThreads, 0, st>>>(c, p, g, partial);
+    } else {
+      auto* c = (const float*)cur;
+      auto* p = (const float*)prev;
+      if (vec)
+        decide_partial_kernel<float, true><<<(unsigned)slabs, kThreads, 0, st>>>(c, p, g, partial);
+      else
+        decide_partial_kernel<float, false><<<(unsigned)slabs, kThreads, 0, st>>>(c, p, g, partial);
+    }
+    FC_LAUNCH_CHECK("decide_partial_kernel");
+  }
+  decide_finalize_kernel<<<1, 1024, 0, st>>>(g, partial, chunk_step, warmup_m, eps, force, acc, l1rel,
+                                             recompute, active_ids, n_active);
+  FC_LAUNCH_CHECK("decide_finalize_kernel");
+  return FC_OK;
+}

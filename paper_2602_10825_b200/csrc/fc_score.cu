@@ -1,0 +1,346 @@
+// fc_kv_score: importance (Eq. 9), max-pool (Eq. 10), redundancy (Eq. 11, through the mean-key
+// identity of the paper's efficiency appendix) and the mixed score (Eq. 12).
+//
+// CUDA-core pipeline, deterministic (no floating-point atomics), five launches per call:
+//   pass1     one thread per key: raw logits of all observation queries against its key,
+//             written to the workspace; normalised key summed per 128-key tile (mean key)
+//   row_lse   one block per (head, query): log-sum-exp of that query's logits over all keys
+//   mean_key  one block per head: tile sums -> mean normalised key
+//   pass2     one thread per key: attention mass of the key (mean over queries of
+//             exp(logit - lse)), and its redundancy logit a_j = meankey.khat_j - |khat_j|^2/L_k;
+//             per-tile softmax statistics of a
+//   finalize  softmax of a over the head, max-pool of the importance, lambda-mix
+#include <cmath>
+
+#include "fc_common.cuh"
+
+namespace {
+
+constexpr int kTile = 128;  // keys per block, one thread each
+
+template <typename T, int D>
+__device__ __forceinline__ void load_row(const T* __restrict__ row, float (&x)[D]) {
+  if constexpr (sizeof(T) == 2) {
+#pragma unroll
+    for (int v = 0; v < D / 8; ++v) {
+      const uint4 w = *reinterpret_cast<const uint4*>(row + v * 8);
+      const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        x[v * 8 + 2 * i] = fc::bf16_lo(ww[i]);
+        x[v * 8 + 2 * i + 1] = fc::bf16_hi(ww[i]);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int v = 0; v < D / 4; ++v) {
+      const float4 w = *reinterpret_cast<const float4*>(row + v * 4);
+      x[v * 4] = w.x;
+      x[v * 4 + 1] = w.y;
+      x[v * 4 + 2] = w.z;
+      x[v * 4 + 3] = w.w;
+    }
+  }
+}
+
+struct ScoreGeom {
+  int H_q, H_kv, d, L_q, L_k, group, n_q, n_tiles;
+  int64_t q_hs, q_rs, k_hs, k_rs;
+  float scale, lambda;
+  int pool_k;
+};
+
+// smem: q_s [n_q][D] then khat_s [kTile][D+1]
+template <typename T, int D>
+__global__ void __launch_bounds__(kTile)
+score_pass1_kernel(const T* __restrict__ Q, const T* __restrict__ K, ScoreGeom g,
+                   float* __restrict__ S, float* __restrict__ mk_partial) {
+  extern __shared__ float sm[];
+  float* q_s = sm;
+  float* khat_s = sm + (size_t)g.n_q * D;
+  const int hk = blockIdx.y, tile = blockIdx.x, tid = threadIdx.x;
+  for (int t = tid; t < g.n_q * D; t += kTile) {
+    const int i = t / D, e = t % D;
+    const int hq = hk * g.group + i / g.L_q, r = i % g.L_q;
+    q_s[t] = fc::to_float(Q[(int64_t)hq * g.q_hs + (int64_t)r * g.q_rs + e]);
+  }
+  const int j = tile * kTile + tid;
+  const bool valid = j < g.L_k;
+  float k[D];
+  if (valid) {
+    load_row<T, D>(K + (int64_t)hk * g.k_hs + (int64_t)j * g.k_rs, k);
+  } else {
+#pragma unroll
+    for (int e = 0; e < D; ++e) k[e] = 0.f;
+  }
+  float n2 = 0.f;
+#pragma unroll
+  for (int e = 0; e < D; ++e) n2 = fmaf(k[e], k[e], n2);
+  const float inv = valid ? 1.f / fmaxf(sqrtf(n2), 1e-12f) : 0.f;
+#pragma unroll
+  for (int e = 0; e < D; ++e) khat_s[tid * (D + 1) + e] = k[e] * inv;
+  __syncthreads();
+  if (valid) {
+    float* s_out = S + ((int64_t)hk * g.n_q) * g.L_k + j;
+    for (int i = 0; i < g.n_q; ++i) {
+      const float4* q4 = reinterpret_cast<const float4*>(q_s + i * D);
+      float dot = 0.f;
+#pragma unroll
+      for (int v = 0; v < D / 4; ++v) {
+        const float4 q = q4[v];
+        dot = fmaf(q.x, k[4 * v], dot);
+        dot = fmaf(q.y, k[4 * v + 1], dot);
+        dot = fmaf(q.z, k[4 * v + 2], dot);
+        dot = fmaf(q.w, k[4 * v + 3], dot);
+      }
+      s_out[(int64_t)i * g.L_k] = dot * g.scale;
+    }
+  }
+  if (tid < D) {
+    float acc = 0.f;
+    for (int r = 0; r < kTile; ++r) acc += khat_s[r * (D + 1) + tid];
+    mk_partial[((int64_t)hk * g.n_tiles + tile) * D + tid] = acc;
+  }
+}
+
+// Fixed-tree block reduction of an online-softmax pair (m, l); result valid in thread 0.
+template <int kThreads>
+__device__ __forceinline__ void reduce_ml(float& m, float& l, float* sm_m, float* sm_l) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float m2 = __shfl_down_sync(0xffffffffu, m, o), l2 = __shfl_down_sync(0xffffffffu, l, o);
+    const float mn = fmaxf(m, m2);
+    l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
+    m = mn;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) {
+    sm_m[warp] = m;
+    sm_l[warp] = l;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    m = sm_m[0];
+    l = sm_l[0];
+    for (int w = 1; w < kThreads / 32; ++w) {
+      const float m2 = sm_m[w], l2 = sm_l[w];
+      const float mn = fmaxf(m, m2);
+      l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
+      m = mn;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+score_row_lse_kernel(const float* __restrict__ S, int L_k, float* __restrict__ lse) {
+  __shared__ float sm_m[8], sm_l[8];
+  const int64_t row = (int64_t)blockIdx.y * gridDim.x + blockIdx.x;  // (head, query)
+  const float* s = S + row * L_k;
+  float m = -INFINITY, l = 0.f;
+  for (int j = threadIdx.x; j < L_k; j += 256) {
+    const float x = s[j];
+    if (x > m) {
+      l = l * expf(m - x) + 1.f;  // expf(-inf) = 0 on the first element
+      m = x;
+    } else {
+      l += expf(x - m);
+    }
+  }
+  reduce_ml<256>(m, l, sm_m, sm_l);
+  if (threadIdx.x == 0) lse[row] = m + logf(l);
+}
+
+__global__ void score_mean_key_kernel(const float* __restrict__ mk_partial, int n_tiles, int d, int L_k,
+                                      float* __restrict__ mean_key) {
+  const int hk = blockIdx.x, e = threadIdx.x;
+  if (e >= d) return;
+  float acc = 0.f;
+  for (int t = 0; t < n_tiles; ++t) acc += mk_partial[((int64_t)hk * n_tiles + t) * d + e];
+  mean_key[hk * d + e] = acc / (float)L_k;
+}
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kTile)
+score_pass2_kernel(const T* __restrict__ K, ScoreGeom g, const float* __restrict__ S,
+                   const float* __restrict__ lse, const float* __restrict__ mean_key,
+                   float* __restrict__ imp_accum, int accum_phase, int n_steps,
+                   float* __restrict__ imp_out, float* __restrict__ a_out, float2* __restrict__ a_partial) {
+  __shared__ float mk_s[D];
+  __shared__ float lse_s[128];
+  __shared__ float sm_m[kTile / 32], sm_l[kTile / 32];
+  const int hk = blockIdx.y, tile = blockIdx.x, tid = threadIdx.x;
+  if (tid < D) mk_s[tid] = mean_key[hk * D + tid];
+  if (tid < g.n_q) lse_s[tid] = lse[hk * g.n_q + tid];
+  __syncthreads();
+  const int j = tile * kTile + tid;
+  const bool valid = j < g.L_k;
+  float a = -INFINITY;
+  if (valid) {
+    const float* s = S + ((int64_t)hk * g.n_q) * g.L_k + j;
+    float mass = 0.f;
+    for (int i = 0; i < g.n_q; ++i) mass += expf(s[(int64_t)i * g.L_k] - lse_s[i]);
+    mass /= (float)g.n_q;
+    const int64_t o = (int64_t)hk * g.L_k + j;
+    if (accum_phase == 1) {
+      imp_accum[o] += mass;
+    } else if (accum_phase == 2) {
+      const float t = imp_accum[o] + mass;
+      imp_accum[o] = t;
+      imp_out[o] = t / (float)n_steps;
+    } else {
+      imp_out[o] = mass;
+    }
+    if (accum_phase != 1) {
+      float k[D];
+      load_row<T, D>(K + (int64_t)hk * g.k_hs + (int64_t)j * g.k_rs, k);
+      float n2 = 0.f, dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < D; ++e) {
+        n2 = fmaf(k[e], k[e], n2);
+        dot = fmaf(mk_s[e], k[e], dot);
+      }
+      const float inv = 1.f / fmaxf(sqrtf(n2), 1e-12f);
+      a = dot * inv - (n2 * inv * inv) / (float)g.L_k;
+      a_out[o] = a;
+    }
+  }
+  if (accum_phase == 1) return;
+  float m = a, l = valid ? 1.f : 0.f;
+  reduce_ml<kTile>(m, l, sm_m, sm_l);
+  if (tid == 0) a_partial[hk * g.n_tiles + tile] = make_float2(m, l);
+}
+
+__global__ void __launch_bounds__(kTile)
+score_finalize_kernel(ScoreGeom g, const float* __restrict__ imp_in, const float* __restrict__ a_in,
+                      const float2* __restrict__ a_partial, float* __restrict__ red_out,
+                      float* __restrict__ score) {
+  __shared__ float sm_m[kTile / 32], sm_l[kTile / 32];
+  __shared__ float sh_m, sh_l;
+  const int hk = blockIdx.y, tile = blockIdx.x, tid = threadIdx.x;
+  float m = -INFINITY, l = 0.f;
+  for (int t = tid; t < g.n_tiles; t += kTile) {
+    const float2 p = a_partial[hk * g.n_tiles + t];
+    const float mn = fmaxf(m, p.x);
+    l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * expf(p.x - mn));
+    m = mn;
+  }
+  reduce_ml<kTile>(m, l, sm_m, sm_l);
+  if (tid == 0) {
+    sh_m = m;
+    sh_l = l;
+  }
+  __syncthreads();
+  const int j = tile * kTile + tid;
+  if (j >= g.L_k) return;
+  const int64_t base = (int64_t)hk * g.L_k;
+  const float red = expf(a_in[base + j] - sh_m) / sh_l;
+  const int half = g.pool_k / 2;
+  float pooled = -INFINITY;
+  for (int u = max(j - half, 0); u <= min(j + half, g.L_k - 1); ++u) pooled = fmaxf(pooled, imp_in[base + u]);
+  if (red_out) red_out[base + j] = red;
+  score[base + j] = g.lambda * pooled - (1.f - g.lambda) * red;
+}
+
+struct ScoreWs {
+  float *S, *mk_partial, *lse, *mean_key, *a, *imp_tmp;
+  float2* a_partial;
+  size_t total;
+};
+
+ScoreWs carve(const ScoreGeom& g, void* ws) {
+  ScoreWs w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* p = ws ? (char*)ws + off : nullptr;
+    off += fc::align_up(bytes, 256);
+    return p;
+  };
+  w.S = (float*)take((size_t)g.H_kv * g.n_q * g.L_k * 4);
+  w.mk_partial = (float*)take((size_t)g.H_kv * g.n_tiles * g.d * 4);
+  w.lse = (float*)take((size_t)g.H_kv * g.n_q * 4);
+  w.mean_key = (float*)take((size_t)g.H_kv * g.d * 4);
+  w.a = (float*)take((size_t)g.H_kv * g.L_k * 4);
+  w.imp_tmp = (float*)take((size_t)g.H_kv * g.L_k * 4);
+  w.a_partial = (float2*)take((size_t)g.H_kv * g.n_tiles * 8);
+  w.total = off;
+  return w;
+}
+
+int make_geom(const fc_score_desc* d, ScoreGeom& g) {
+  if (!d) return FC_ERR_INVALID_ARG;
+  if (d->H_q <= 0 || d->H_kv <= 0 || d->H_q % d->H_kv || d->L_q <= 0 || d->L_k <= 0) return FC_ERR_INVALID_ARG;
+  if (d->pool_k < 1 || d->pool_k % 2 == 0) return FC_ERR_INVALID_ARG;
+  if (d->d != 64 && d->d != 128) return FC_ERR_UNSUPPORTED;
+  g.H_q = d->H_q; g.H_kv = d->H_kv; g.d = d->d; g.L_q = d->L_q; g.L_k = d->L_k;
+  g.group = d->H_q / d->H_kv;
+  g.n_q = g.group * d->L_q;
+  if (g.n_q > 128) return FC_ERR_UNSUPPORTED;
+  g.n_tiles = (d->L_k + kTile - 1) / kTile;
+  g.q_hs = d->q_hs; g.q_rs = d->q_rs; g.k_hs = d->k_hs; g.k_rs = d->k_rs;
+  g.scale = d->scale != 0.f ? d->scale : 1.f / sqrtf((float)d->d);
+  g.lambda = d->lambda;
+  g.pool_k = d->pool_k;
+  return FC_OK;
+}
+
+template <typename T, int D>
+int run(cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, const void* K,
+        float* imp_accum, int phase, int n_steps, float* imp, float* red, float* score) {
+  const size_t smem1 = ((size_t)g.n_q * D + (size_t)kTile * (D + 1)) * 4;
+  FC_CUDA_CHECK(cudaFuncSetAttribute(score_pass1_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem1));
+  dim3 grid(g.n_tiles, g.H_kv);
+  score_pass1_kernel<T, D><<<grid, kTile, smem1, st>>>((const T*)Q, (const T*)K, g, w.S, w.mk_partial);
+  FC_LAUNCH_CHECK("score_pass1_kernel");
+  score_row_lse_kernel<<<dim3(g.n_q, g.H_kv), 256, 0, st>>>(w.S, g.L_k, w.lse);
+  FC_LAUNCH_CHECK("score_row_lse_kernel");
+  score_mean_key_kernel<<<g.H_kv, 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
+  FC_LAUNCH_CHECK("score_mean_key_kernel");
+  float* imp_buf = imp ? imp : w.imp_tmp;
+  score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, w.S, w.lse, w.mean_key, imp_accum, phase,
+                                                   n_steps, imp_buf, w.a, w.a_partial);
+  FC_LAUNCH_CHECK("score_pass2_kernel");
+  if (phase != 1) {
+    score_finalize_kernel<<<grid, kTile, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
+    FC_LAUNCH_CHECK("score_finalize_kernel");
+  }
+  return FC_OK;
+}
+
+}  // namespace
+
+extern "C" size_t fc_kv_score_workspace_bytes(const fc_score_desc* desc) {
+  ScoreGeom g;
+  if (make_geom(desc, g) != FC_OK) return 0;
+  return carve(g, nullptr).total;
+}
+
+extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc, const void* Q_obs,
+                           const void* K_cand, int dtype, float* imp_accum, int accum_phase, int n_steps,
+                           float* imp, float* red, float* score, uint32_t* status, void* ws,
+                           size_t ws_bytes) {
+  (void)status;
+  if (!ctx || !Q_obs || !K_cand) return FC_ERR_INVALID_ARG;
+  ScoreGeom g;
+  int rc = make_geom(desc, g);
+  if (rc != FC_OK) return rc;
+  if (dtype != FC_BF16 && dtype != FC_F32) return FC_ERR_UNSUPPORTED;
+  if (accum_phase < 0 || accum_phase > 2) return FC_ERR_INVALID_ARG;
+  if (accum_phase != 0 && (!imp_accum || n_steps <= 0)) return FC_ERR_INVALID_ARG;
+  if (accum_phase != 1 && !score) return FC_ERR_INVALID_ARG;
+  const int es = fc::elem_size(dtype);
+  if (!fc::aligned16(Q_obs) || !fc::aligned16(K_cand)) return FC_ERR_MISALIGNED;
+  if ((g.k_hs * es) % 16 || (g.k_rs * es) % 16 || (g.q_hs * es) % 16 || (g.q_rs * es) % 16)
+    return FC_ERR_MISALIGNED;
+  if (g.k_rs < g.d || g.q_rs < g.d) return FC_ERR_INVALID_ARG;
+  const ScoreWs w = carve(g, ws);
+  if (!ws || ws_bytes < w.total) return FC_ERR_WORKSPACE;
+  if (!fc::aligned16(ws)) return FC_ERR_MISALIGNED;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (dtype == FC_BF16) {
+    if (g.d == 128) return run<__nv_bfloat16, 128>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
+    return run<__nv_bfloat16, 64>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
+  }
+  if (g.d == 128) return run<float, 128>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
+  return run<float, 64>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
+}

@@ -1,0 +1,257 @@
+// fc_kv_select_compact: per-head top-B of the selection score (text after Eq. 12) and the
+// retention of the selected K/V rows (Sec. 3.3).
+//
+// Selection: one 1024-thread block per head.  Scores become order-preserving 32-bit keys (NaN
+// ranks as -inf, -0 as +0) held in shared memory when they fit; a 4-pass, 8-bit-digit radix
+// select finds the key T of the B-th largest score and how many keys exceed it; one ordered
+// compaction then keeps every key above T plus the lowest-index keys equal to T, so the kept
+// set is exactly the first B elements of the total order (score descending, index ascending),
+// written in ascending index order.  Integer work only: bit-exact.
+//
+// Compaction: a separate streaming kernel moves whole rows with 16-byte accesses, several
+// independent loads in flight per thread; rows that were dropped are never read.
+#include "fc_common.cuh"
+
+namespace {
+
+constexpr int kSelThreads = 1024;
+
+__device__ __forceinline__ uint32_t score_key(float s, bool& is_nan) {
+  uint32_t u = __float_as_uint(s);
+  is_nan = (u & 0x7fffffffu) > 0x7f800000u;
+  if (is_nan) u = 0xff800000u;              // -inf
+  if ((u << 1) == 0) u = 0;                 // -0 -> +0
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // larger float <=> larger key
+}
+
+template <bool kSmemKeys>
+__global__ void __launch_bounds__(kSelThreads)
+select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __restrict__ kept_idx,
+                   uint32_t* __restrict__ status) {
+  extern __shared__ uint32_t smem_keys[];
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t sh_prefix, sh_remaining, sh_nan;
+  const int h = blockIdx.x, tid = threadIdx.x;
+  const float* s = score + (size_t)h * L_k;
+  int32_t* out = kept_idx + (size_t)h * B;  // B <= L_k here (the identity case is handled apart)
+
+  if (tid == 0) sh_nan = 0;
+  __syncthreads();
+  bool any_nan = false;
+  if (kSmemKeys) {
+    for (int j = tid; j < L_k; j += kSelThreads) {
+      bool n;
+      smem_keys[j] = score_key(s[j], n);
+      any_nan |= n;
+    }
+  }
+  auto key_at = [&](int j) -> uint32_t {
+    if (kSmemKeys) return smem_keys[j];
+    bool n;
+    uint32_t k = score_key(s[j], n);
+    any_nan |= n;
+    return k;
+  };
+
+  // Radix select, most significant digit first.  Invariant: the B-th largest key has the bits
+  // of `prefix` in the digits already fixed, and `remaining` of the keys with that prefix
+  // (counted from the largest) are still to be taken.
+  uint32_t prefix = 0, prefix_mask = 0, remaining = (uint32_t)B;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    for (int j = tid; j < L_k; j += kSelThreads) {
+      const uint32_t k = key_at(j);
+      if ((k & prefix_mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t rem = remaining;
+      int digit = 255;
+      for (; digit > 0; --digit) {
+        if (hist[digit] >= rem) break;
+        rem -= hist[digit];
+      }
+      sh_prefix = prefix | ((uint32_t)digit << shift);
+      sh_remaining = rem;
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    remaining = sh_remaining;
+    prefix_mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t T = prefix;           // key of the B-th largest score
+  const uint32_t need_eq = remaining;  // how many keys equal to T are kept (lowest indices)
+
+  // Ordered compaction: thread t owns the contiguous index range [t*per, (t+1)*per).
+  const int per = (L_k + kSelThreads - 1) / kSelThreads;
+  const int j0 = min(tid * per, L_k), j1 = min(j0 + per, L_k);
+  uint32_t n_gt = 0, n_eq = 0;
+  for (int j = j0; j < j1; ++j) {
+    const uint32_t k = key_at(j);
+    n_gt += k > T;
+    n_eq += k == T;
+  }
+  // exclusive block scan of the packed pair (eq in the high half, gt in the low half)
+  uint32_t packed = (n_eq << 16) | n_gt;  // per-thread counts < 65536 (L_k/1024 items per thread)
+  uint32_t incl = packed;
+  const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  // a warp's totals stay below 2^16 per half (L_k <= 2^20); block-level bases use full words
+  __shared__ uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32];
+  if (lane == 31) {
+    warp_gt[warp] = incl & 0xffffu;
+    warp_eq[warp] = incl >> 16;
+  }
+  __syncthreads();
+  uint32_t base_gt = 0, base_eq = 0;
+  for (int w = 0; w < warp; ++w) {
+    base_gt += warp_gt[w];
+    base_eq += warp_eq[w];
+  }
+  uint32_t gt_before = base_gt + (incl & 0xffffu) - n_gt;
+  uint32_t eq_before = base_eq + (incl >> 16) - n_eq;
+  for (int j = j0; j < j1; ++j) {
+    const uint32_t k = key_at(j);
+    if (k > T) {
+      out[gt_before + min(eq_before, need_eq)] = j;
+      ++gt_before;
+    } else if (k == T) {
+      if (eq_before < need_eq) out[gt_before + eq_before] = j;
+      ++eq_before;
+    }
+  }
+  if (any_nan) sh_nan = 1;
+  __syncthreads();
+  if (tid == 0 && sh_nan && status) atomicOr(status, FC_DEV_NAN_SCORE);
+}
+
+__global__ void select_identity_kernel(int32_t* __restrict__ kept_idx, int n_heads, int L_k,
+                                       const float* __restrict__ score, uint32_t* __restrict__ status) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (int64_t)n_heads * L_k) return;
+  kept_idx[i] = (int32_t)(i % L_k);
+  if (status) {
+    const uint32_t u = __float_as_uint(score[i]);
+    if ((u & 0x7fffffffu) > 0x7f800000u) atomicOr(status, FC_DEV_NAN_SCORE);
+  }
+}
+
+__global__ void write_count_kernel(int32_t* n_kept, int32_t v) { *n_kept = v; }
+
+// Row gather.  The copy of one head is a flat list of 16-byte pieces: piece p of the head
+// belongs to kept row p / pieces_per_row.  A block moves kUnroll * blockDim pieces of K and of V;
+// all loads of a thread are issued before its first store.
+constexpr int kCopyThreads = 256;
+constexpr int kUnroll = 4;
+
+__global__ void __launch_bounds__(kCopyThreads)
+gather_rows_kernel(const uint8_t* __restrict__ K_src, const uint8_t* __restrict__ V_src,
+                   uint8_t* __restrict__ K_dst, uint8_t* __restrict__ V_dst,
+                   const int32_t* __restrict__ kept_idx, int n_keep, int L_k, int pieces_per_row,
+                   int64_t src_hs_b, int64_t src_rs_b, int64_t dst_hs_b, int64_t dst_rs_b,
+                   uint32_t* __restrict__ status) {
+  const int h = blockIdx.y;
+  const int64_t n_pieces = (int64_t)n_keep * pieces_per_row;
+  const int64_t p0 = (int64_t)blockIdx.x * (kCopyThreads * kUnroll) + threadIdx.x;
+  const int32_t* idx = kept_idx + (size_t)h * n_keep;
+  uint4 kv[kUnroll], vv[kUnroll];
+  int64_t dst_off[kUnroll];
+  bool ok[kUnroll];
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u) {
+    const int64_t p = p0 + (int64_t)u * kCopyThreads;
+    ok[u] = p < n_pieces;
+    if (ok[u]) {
+      const int r = (int)(p / pieces_per_row), c = (int)(p % pieces_per_row);
+      const int32_t src_row = idx[r];
+      if (src_row < 0 || src_row >= L_k) {  // never produced by the selection kernel
+        ok[u] = false;
+        if (status) atomicOr(status, FC_DEV_BAD_INDEX);
+        continue;
+      }
+      const int64_t so = (int64_t)h * src_hs_b + (int64_t)src_row * src_rs_b + c * 16;
+      dst_off[u] = (int64_t)h * dst_hs_b + (int64_t)r * dst_rs_b + c * 16;
+      kv[u] = fc::ld_stream16(K_src + so);
+      vv[u] = fc::ld_stream16(V_src + so);
+    }
+  }
+#pragma unroll
+  for (int u = 0; u < kUnroll; ++u)
+    if (ok[u]) {
+      fc::st_stream16(K_dst + dst_off[u], kv[u]);
+      fc::st_stream16(V_dst + dst_off[u], vv[u]);
+    }
+}
+
+constexpr size_t kStaticSelSmem = 256 * 4 + 3 * (kSelThreads / 32) * 4 + 64;
+
+}  // namespace
+
+extern "C" size_t fc_kv_select_compact_workspace_bytes(int n_heads, int L_k) {
+  (void)n_heads;
+  (void)L_k;
+  return 16;  // the selection works in shared memory; a token size keeps the calling convention uniform
+}
+
+extern "C" int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* score, int n_heads, int L_k,
+                                    int B, const void* K_src, const void* V_src, void* K_dst, void* V_dst,
+                                    int dtype, int d, const fc_compact_strides* strides, int32_t* kept_idx,
+                                    int32_t* n_kept, uint32_t* status, void* ws, size_t ws_bytes) {
+  (void)ws;
+  (void)ws_bytes;
+  if (!ctx || !score || !kept_idx || n_heads <= 0 || L_k <= 0 || B <= 0) return FC_ERR_INVALID_ARG;
+  const bool copy = K_src || V_src || K_dst || V_dst;
+  if (copy) {
+    if (!K_src || !V_src || !K_dst || !V_dst || !strides) return FC_ERR_INVALID_ARG;
+    if (dtype != FC_BF16 && dtype != FC_F32) return FC_ERR_UNSUPPORTED;
+    if (d <= 0) return FC_ERR_INVALID_ARG;
+    const int es = fc::elem_size(dtype);
+    if ((d * es) % 16) return FC_ERR_UNSUPPORTED;
+    if (!fc::aligned16(K_src) || !fc::aligned16(V_src) || !fc::aligned16(K_dst) || !fc::aligned16(V_dst))
+      return FC_ERR_MISALIGNED;
+    const int64_t st[4] = {strides->src_hs, strides->src_rs, strides->dst_hs, strides->dst_rs};
+    for (int i = 0; i < 4; ++i)
+      if (st[i] < 0 || (st[i] * es) % 16) return FC_ERR_MISALIGNED;
+    if (strides->src_rs < d || strides->dst_rs < d) return FC_ERR_INVALID_ARG;
+  }
+  if (L_k > (1 << 20)) return FC_ERR_UNSUPPORTED;  // keeps the packed 16-bit scan counters exact
+  cudaStream_t st = (cudaStream_t)stream;
+  const int n_keep = B < L_k ? B : L_k;
+  if (B >= L_k) {
+    const int64_t n = (int64_t)n_heads * L_k;
+    select_identity_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kept_idx, n_heads, L_k, score, status);
+    FC_LAUNCH_CHECK("select_identity_kernel");
+  } else {
+    const size_t key_bytes = (size_t)L_k * 4;
+    if (key_bytes + kStaticSelSmem + 1024 <= (size_t)ctx->smem_optin) {
+      FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+      select_topb_kernel<true><<<n_heads, kSelThreads, key_bytes, st>>>(score, L_k, B, kept_idx, status);
+    } else {
+      select_topb_kernel<false><<<n_heads, kSelThreads, 0, st>>>(score, L_k, B, kept_idx, status);
+    }
+    FC_LAUNCH_CHECK("select_topb_kernel");
+  }
+  if (n_kept) {
+    write_count_kernel<<<1, 1, 0, st>>>(n_kept, n_keep);
+    FC_LAUNCH_CHECK("write_count_kernel");
+  }
+  if (copy) {
+    const int es = fc::elem_size(dtype);
+    const int ppr = d * es / 16;
+    const int64_t n_pieces = (int64_t)n_keep * ppr;
+    dim3 grid((unsigned)((n_pieces + kCopyThreads * kUnroll - 1) / (kCopyThreads * kUnroll)), n_heads);
+    gather_rows_kernel<<<grid, kCopyThreads, 0, st>>>(
+        (const uint8_t*)K_src, (const uint8_t*)V_src, (uint8_t*)K_dst, (uint8_t*)V_dst, kept_idx, n_keep,
+        L_k, ppr, strides->src_hs * es, strides->src_rs * es, strides->dst_hs * es, strides->dst_rs * es,
+        status);
+    FC_LAUNCH_CHECK("gather_rows_kernel");
+  }
+  return FC_OK;
+}

@@ -1,0 +1,372 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, on the same seeded inputs.
+
+Bars: decisions, active lists and kept indices bit-exact; compacted rows byte-exact; fp32 outputs
+within 1e-4; bf16 attention within max-abs 1e-2 and relative-L2 1e-2; importance / redundancy /
+score within 1e-4 of the row maximum.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2602_10825_b200 as fc
+    from paper_2602_10825_b200 import build as fc_build
+    fc_build.build()
+    c = fc.Context(0)
+    yield c
+    c.close()
+
+
+def dev(t):
+    return t.cuda()
+
+
+def i32(x):
+    return torch.as_tensor(np.asarray(x), dtype=torch.int32).cuda()
+
+
+# ------------------------------------------------------------------------------------ decide
+
+def _run_decide_sequence(ctx, dtype, lens, n_steps, eps, m, seed, r_hi=0.2):
+    n = len(lens)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    acc_o = np.zeros(n, np.float32)
+    acc_g = torch.zeros(n, dtype=torch.float32, device="cuda")
+    min_margin = math.inf
+    for s in range(n_steps):
+        target = wl.uniform((n,), seed * 100 + s, 0.0, r_hi)
+        parts = [wl.indicator_pair(1, int(L), [float(target[c])], seed * 1000 + s * 10 + c, dtype=dtype)
+                 for c, L in enumerate(lens)]
+        cur = torch.cat([p[0] for p in parts])
+        prev = torch.cat([p[1] for p in parts])
+        step = np.full(n, s, np.int32)
+        want = oracle.chunk_decide(wl.bits(cur), wl.bits(prev), off, step, m, eps, acc_o)
+        margin = np.abs(acc_o + want["l1rel"] - eps)
+        min_margin = min(min_margin, float(margin[step >= m].min()) if (step >= m).any() else math.inf)
+        got = ctx.chunk_decide(dev(cur), dev(prev), off, i32(step), m, eps, acc_g)
+        torch.cuda.synchronize()
+        assert got["recompute"].cpu().numpy().tolist() == want["recompute"].tolist(), f"step {s}"
+        assert int(got["n_active"].item()) == want["n_active"]
+        ids = got["active_ids"].cpu().numpy()
+        assert ids[:want["n_active"]].tolist() == want["active_ids"].tolist()
+        assert (ids[want["n_active"]:] == -1).all()
+        np.testing.assert_allclose(got["l1rel"].cpu().numpy(), want["l1rel"], rtol=2e-6)
+        np.testing.assert_allclose(acc_g.cpu().numpy(), want["acc"], rtol=4e-6, atol=1e-9)
+        acc_o = want["acc"]
+    # the decisions above are only meaningful if no step sat on the threshold
+    assert min_margin > 1e-3 * eps, f"a step came within {min_margin} of eps; change the seed"
+
+
+def test_decide_tiny_f32_config(ctx):
+    w = wl.CONFIGS["tiny_f32"]
+    _run_decide_sequence(ctx, torch.float32, [w.n_c * w.hidden] * w.W, w.n_steps, w.eps, w.warmup_m, w.seed)
+
+
+def test_decide_bf16_ragged_and_unaligned(ctx):
+    # lengths that are not multiples of the slab, of the vector, or aligned to 16 bytes
+    _run_decide_sequence(ctx, torch.bfloat16, [8192 * 3 + 8, 40000, 8, 123456], 4, 0.1, 1, 7)
+    _run_decide_sequence(ctx, torch.bfloat16, [1001, 77777, 3], 3, 0.1, 1, 8)
+    _run_decide_sequence(ctx, torch.float32, [4099, 65536 + 4, 5], 3, 0.1, 2, 9)
+
+
+def test_decide_special_cases(ctx):
+    n = 4096
+    prev = torch.ones(2 * n)
+    cur = torch.full((2 * n,), 1.25)
+    cur[n:] = 0.0
+    prev[n:] = 0.0  # second chunk: zero over zero -> r = 0
+    off = [0, n, 2 * n]
+    acc = torch.zeros(2, device="cuda")
+    out = ctx.chunk_decide(dev(cur), dev(prev), off, i32([3, 3]), 1, 0.25, acc)
+    assert out["recompute"].cpu().tolist() == [0, 0]  # s == eps reuses (strict >)
+    assert out["l1rel"].cpu().tolist() == [0.25, 0.0]
+    cur[n:] = 1.0  # zero denominator, positive numerator -> +inf -> recompute
+    acc.zero_()
+    out = ctx.chunk_decide(dev(cur), dev(prev), off, i32([3, 3]), 1, 10.0, acc)
+    assert out["recompute"].cpu().tolist() == [0, 1] and math.isinf(out["l1rel"][1].item())
+    # forced chunk and warm-up reset the accumulator
+    acc.fill_(0.2)
+    out = ctx.chunk_decide(dev(cur), dev(prev), off, i32([0, 9]), 1, 1e9, acc,
+                           force=torch.tensor([0, 1], dtype=torch.uint8).cuda())
+    assert out["recompute"].cpu().tolist() == [1, 1] and acc.cpu().tolist() == [0.0, 0.0]
+    # run-to-run bit reproducibility
+    cur2, prev2 = wl.indicator_pair(3, 100000, [0.1, 0.2, 0.3], 3)
+    a = ctx.chunk_decide(dev(cur2), dev(prev2), [0, 100000, 200000, 300000], i32([5] * 3), 1, 0.5,
+                         torch.zeros(3, device="cuda"))["l1rel"].clone()
+    b = ctx.chunk_decide(dev(cur2), dev(prev2), [0, 100000, 200000, 300000], i32([5] * 3), 1, 0.5,
+                         torch.zeros(3, device="cuda"))["l1rel"]
+    assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("name", ["cached_step_bf16"])
+def test_decide_full_size(ctx, name):
+    w = wl.CONFIGS[name]
+    lens = [w.n_c * w.hidden] * w.W
+    _run_decide_sequence(ctx, w.torch_dtype, lens, 2, 0.1, 1, w.seed)
+
+
+# ------------------------------------------------------------------------------------ attention
+
+def _attention_case(ctx, w, active, *, impl=0, token_map=False, sample=None, atol, rel_l2, check_lse=True):
+    Q, K, V = wl.qkv(w)
+    q_off, vis, slo, spo = wl.prefix_layout(w)
+    O0 = wl.normal((w.H, w.window_rows, w.d), 999, 1.0, w.torch_dtype)  # "cached outputs" of earlier steps
+    Og = dev(O0).clone()
+    lse_g = torch.full((w.H, w.window_rows), float("nan"), device="cuda")
+    tok = None
+    kw = {}
+    if token_map:
+        rng = np.random.default_rng(w.seed)
+        L = K.shape[1]
+        tok = np.stack([rng.permutation(L) for _ in range(w.H)]).astype(np.int32)
+        K2, V2 = torch.empty_like(K), torch.empty_like(V)
+        for h in range(w.H):
+            K2[h, tok[h]] = K[h]
+            V2[h, tok[h]] = V[h]
+        K, V = K2, V2
+        kw["kv_token_index"] = i32(tok)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    n_act = i32([len(active)])
+    act = i32(list(active) + [-1] * (w.W - len(active)))
+    ctx.chunk_attention(dev(Q), dev(K), dev(V), q_off, vis, None if token_map else slo,
+                        None if token_map else spo, act, n_act, Og, lse=lse_g, impl=impl, status=status, **kw)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    O_want, lse_want = oracle.chunk_attention(
+        wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, None if token_map else slo,
+        None if token_map else spo, active, kv_token_index=tok, sample_rows=sample,
+        O_init=None if sample is not None else O0.double().numpy())
+    got = Og.double().cpu().numpy()
+    lse_got = lse_g.double().cpu().numpy()
+    if sample is not None:
+        rows = np.asarray(sample)
+        is_act = np.isin(rows // w.n_c, list(active))
+        got_s, want_s = got[:, rows[is_act]], O_want[:, is_act]
+        lse_got_s, lse_want_s = lse_got[:, rows[is_act]], lse_want[:, is_act]
+    else:
+        rows_act = np.concatenate([np.arange(q_off[c], q_off[c + 1]) for c in active]) if active else np.array([], int)
+        got_s, want_s = got[:, rows_act], O_want[:, rows_act]
+        lse_got_s, lse_want_s = lse_got[:, rows_act], lse_want[:, rows_act]
+    if got_s.size:
+        assert np.abs(got_s - want_s).max() <= atol
+        assert np.linalg.norm(got_s - want_s) <= rel_l2 * np.linalg.norm(want_s)
+        if check_lse:
+            np.testing.assert_allclose(lse_got_s, lse_want_s, atol=2e-3 if w.dtype == "bf16" else 1e-4)
+    # rows of chunks that were not recomputed keep their cached values, bit for bit
+    inactive = [c for c in range(w.W) if c not in active]
+    for c in inactive:
+        assert torch.equal(Og[:, q_off[c]:q_off[c + 1]].cpu(), O0[:, q_off[c]:q_off[c + 1]])
+        assert torch.isnan(lse_g[:, q_off[c]:q_off[c + 1]]).all()
+    return Og
+
+
+def test_attention_tiny_f32_config_every_element(ctx):
+    w = wl.CONFIGS["tiny_f32"]
+    _attention_case(ctx, w, [0, 1, 2, 3], atol=1e-4, rel_l2=1e-4)
+    _attention_case(ctx, w, [1, 3], atol=1e-4, rel_l2=1e-4)
+
+
+def test_attention_all_skip_returns_cached_outputs(ctx):
+    w = wl.CONFIGS["tiny_f32"]
+    _attention_case(ctx, w, [], atol=0, rel_l2=0)
+
+
+@pytest.mark.parametrize("dtype,d", [("f32", 128), ("bf16", 64), ("bf16", 128)])
+def test_attention_simt_ragged(ctx, dtype, d):
+    # chunk length 200 = 6 row-tiles of 32 + 8; budget 77 (not a multiple of the key tile)
+    w = wl.Workload("r", dtype, H=3, d=d, W=3, n_c=200, B=77, L_k=277, seed=12, sigma=0.7)
+    tol = dict(atol=1e-4, rel_l2=1e-4) if dtype == "f32" else dict(atol=1e-2, rel_l2=1e-2)
+    _attention_case(ctx, w, [0, 2], impl=1, **tol)
+
+
+def test_attention_token_index_map(ctx):
+    w = wl.Workload("m", "f32", H=2, d=64, W=2, n_c=96, B=50, L_k=146, seed=13)
+    _attention_case(ctx, w, [0, 1], token_map=True, atol=1e-4, rel_l2=1e-4)
+    wb = wl.Workload("m", "bf16", H=2, d=128, W=2, n_c=96, B=50, L_k=146, seed=14, sigma=0.5)
+    _attention_case(ctx, wb, [1], token_map=True, atol=1e-2, rel_l2=1e-2)
+
+
+def test_attention_bf16_tensor_core_small(ctx):
+    # several 128-row tiles with ragged tails in both rows and keys, a clean region and a window
+    w = wl.Workload("t", "bf16", H=2, d=128, W=3, n_c=328, B=200, L_k=528, seed=15, sigma=0.5)
+    _attention_case(ctx, w, [0, 1, 2], atol=1e-2, rel_l2=1e-2)
+    _attention_case(ctx, w, [2], atol=1e-2, rel_l2=1e-2)
+    w2 = wl.Workload("t2", "bf16", H=3, d=128, W=2, n_c=1000, B=0, L_k=1000, seed=16, sigma=0.5)
+    _attention_case(ctx, w2, [0, 1], atol=1e-2, rel_l2=1e-2)
+
+
+def test_attention_bf16_matches_cuda_core_kernel(ctx):
+    # second opinion on the device: tensor-core and CUDA-core kernels agree on a mid-size case
+    w = wl.Workload("x", "bf16", H=4, d=128, W=4, n_c=1160, B=2000, L_k=3160, seed=17, sigma=0.5)
+    a = _attention_case(ctx, w, [0, 2, 3], impl=0, sample=wl.sample_rows(w, 24, 0), atol=1e-2, rel_l2=1e-2)
+    b = _attention_case(ctx, w, [0, 2, 3], impl=1, sample=wl.sample_rows(w, 24, 0), atol=1e-2, rel_l2=1e-2)
+    assert (a.float() - b.float()).abs().max().item() <= 1e-2
+
+
+# ------------------------------------------------------------------------------------ scores
+
+def _score_case(ctx, Q, K, lam, pool_k, impl=0):
+    want = oracle.kv_score(wl.bits(Q), wl.bits(K), lambda_=lam, pool_k=pool_k)
+    H, L = K.shape[0], K.shape[1]
+    imp = torch.empty((H, L), device="cuda")
+    red = torch.empty((H, L), device="cuda")
+    got = ctx.kv_score(dev(Q), dev(K), lambda_=lam, pool_k=pool_k, imp=imp, red=red, impl=impl)
+    torch.cuda.synchronize()
+    for name, g, wnt in (("imp", imp, want["imp"]), ("red", red, want["red"]),
+                         ("score", got["score"], want["score"].astype(np.float64))):
+        g = g.double().cpu().numpy()
+        bound = 1e-4 * np.abs(wnt).max(axis=1, keepdims=True)
+        assert (np.abs(g - wnt) <= bound).all(), name
+    return got["score"], want["score"]
+
+
+def test_score_tiny_f32_config(ctx):
+    w = wl.CONFIGS["tiny_f32"]
+    Q_obs, K, _ = wl.candidates(w)
+    _score_case(ctx, Q_obs, K, w.lam, w.pool_k)
+
+
+@pytest.mark.parametrize("keys", ["normal", "clustered"])
+def test_score_bf16_ragged(ctx, keys):
+    w = wl.Workload("s", "bf16", H=3, d=128, W=1, n_c=100, B=1000, L_k=1331, seed=21, sigma=0.5, keys=keys)
+    Q_obs, K, _ = wl.candidates(w)
+    _score_case(ctx, Q_obs, K, 0.07, 7)
+    _score_case(ctx, Q_obs, K, 0.5, 1)
+
+
+def test_score_gqa_and_d64(ctx):
+    Q = wl.normal((4, 20, 64), 31, 1.0)
+    K = wl.normal((2, 300, 64), 32, 1.0)
+    _score_case(ctx, Q, K, 0.2, 3)
+
+
+def test_score_accumulated_over_steps(ctx):
+    K = wl.normal((2, 700, 128), 41, 0.5, torch.bfloat16)
+    Qs = [wl.normal((2, 50, 128), 42 + s, 0.5, torch.bfloat16) for s in range(3)]
+    acc_o = np.zeros((2, 700), np.float64)
+    acc_g = torch.zeros((2, 700), device="cuda")
+    for s, q in enumerate(Qs):
+        phase = 2 if s == 2 else 1
+        want = oracle.kv_score(wl.bits(q), wl.bits(K), imp_accum=acc_o, accum_phase=phase, n_steps=3)
+        imp = torch.empty((2, 700), device="cuda")
+        got = ctx.kv_score(dev(q), dev(K), imp_accum=acc_g, accum_phase=phase, n_steps=3, imp=imp)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(imp.cpu().numpy(), want["imp"], rtol=0, atol=1e-4 * want["imp"].max())
+    np.testing.assert_allclose(got["score"].cpu().numpy(), want["score"], rtol=0,
+                               atol=1e-4 * np.abs(want["score"]).max())
+
+
+# ------------------------------------------------------------------------------------ select + compact
+
+def _select_case(ctx, score, B, K=None, V=None):
+    want = oracle.kv_select_compact(score, B, None if K is None else wl.bits(K), None if V is None else wl.bits(V))
+    H, L = score.shape
+    n_keep = min(B, L)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    if K is not None:
+        # canaries around the destination: one extra row per head must stay untouched
+        Kd = torch.full((H, n_keep + 1, K.shape[2]), 7.0, dtype=K.dtype, device="cuda")
+        Vd = torch.full((H, n_keep + 1, K.shape[2]), 7.0, dtype=K.dtype, device="cuda")
+        got = ctx.kv_select_compact(torch.from_numpy(score).cuda(), B, dev(K), dev(V), Kd[:, :n_keep], Vd[:, :n_keep],
+                                    status=status)
+    else:
+        got = ctx.kv_select_compact(torch.from_numpy(score).cuda(), B, status=status)
+    torch.cuda.synchronize()
+    assert np.array_equal(got["kept_idx"].cpu().numpy(), want["kept_idx"])
+    assert int(got["n_kept"].item()) == want["n_kept"] == n_keep
+    if K is not None:
+        assert np.array_equal(wl.bits(Kd[:, :n_keep].cpu()), want["K_dst"])
+        assert np.array_equal(wl.bits(Vd[:, :n_keep].cpu()), want["V_dst"])
+        assert (Kd[:, n_keep] == 7.0).all() and (Vd[:, n_keep] == 7.0).all()
+    return status.item()
+
+
+def test_select_bit_exact_with_ties_nan_and_zeros(ctx):
+    rng = np.random.default_rng(5)
+    score = rng.normal(size=(4, 5000)).astype(np.float32)
+    score[:, ::5] = score[:, 2:3]          # one value repeated 1000 times per head
+    score[1, 17] = np.nan
+    score[2, 100:200] = 0.0
+    score[2, 150] = -0.0
+    score[3] = 1.0                          # a head where every score ties
+    for B in (1, 2, 999, 1000, 1001, 2500, 4999, 5000, 6000):
+        st = _select_case(ctx, score, B)
+        assert st & 2  # the NaN was reported
+    assert _select_case(ctx, np.ascontiguousarray(score[2:]), 700) == 0
+
+
+def test_select_compact_tiny_and_ragged(ctx):
+    w = wl.CONFIGS["tiny_f32"]
+    _, K, V = wl.candidates(w)
+    score = oracle.kv_score(wl.bits(wl.candidates(w)[0]), wl.bits(K))["score"]
+    _select_case(ctx, score, w.B, K, V)
+    _select_case(ctx, score, w.L_k, K, V)       # budget = cache length: identity
+    _select_case(ctx, score, w.L_k + 100, K, V)  # budget beyond it: identity
+    wb = wl.Workload("c", "bf16", H=5, d=128, W=1, n_c=10, B=3001, L_k=4099, seed=6, sigma=0.5)
+    _, Kb, Vb = wl.candidates(wb)
+    sb = np.random.default_rng(9).normal(size=(5, 4099)).astype(np.float32)
+    _select_case(ctx, sb, wb.B, Kb, Vb)
+    wc = wl.Workload("c", "bf16", H=2, d=64, W=1, n_c=10, B=100, L_k=333, seed=6, sigma=0.5)
+    _, Kc, Vc = wl.candidates(wc)
+    _select_case(ctx, sb[:2, :333].copy(), 100, Kc, Vc)
+
+
+def test_select_large_head_falls_back_to_global_keys(ctx):
+    rng = np.random.default_rng(11)
+    score = rng.normal(size=(2, 70001)).astype(np.float32)  # 280 KB of keys: beyond shared memory
+    score[:, ::3] = 0.5
+    _select_case(ctx, score, 33333)
+
+
+def test_pipeline_gpu_scores_feed_gpu_select(ctx):
+    # end to end on the device: score -> select on the library's own fp32 scores; the oracle's
+    # selection on those same scores (copied back) must give the same indices
+    w = wl.Workload("p", "bf16", H=4, d=128, W=1, n_c=50, B=1500, L_k=2345, seed=33, sigma=0.5, keys="clustered")
+    Q_obs, K, V = wl.candidates(w)
+    got = ctx.kv_score(dev(Q_obs), dev(K))
+    sel = ctx.kv_select_compact(got["score"], w.B, dev(K), dev(V))
+    torch.cuda.synchronize()
+    want = oracle.kv_select_compact(got["score"].cpu().numpy(), w.B, wl.bits(K), wl.bits(V))
+    assert np.array_equal(sel["kept_idx"].cpu().numpy(), want["kept_idx"])
+    assert np.array_equal(wl.bits(sel["K_dst"].cpu()), want["K_dst"])
+    # information only: overlap with the fully-oracle pipeline
+    full = oracle.kv_select_compact(oracle.kv_score(wl.bits(Q_obs), wl.bits(K))["score"], w.B)
+    overlap = np.mean([len(set(a) & set(b)) / w.B for a, b in zip(full["kept_idx"], want["kept_idx"])])
+    assert overlap > 0.99
+
+
+# ------------------------------------------------------------------------------------ error conventions
+
+def test_bad_arguments_return_a_status_and_launch_nothing(ctx):
+    import paper_2602_10825_b200 as fc
+    w = wl.CONFIGS["tiny_f32"]
+    Q, K, V = (dev(t) for t in wl.qkv(w))
+    q_off, vis, slo, spo = wl.prefix_layout(w)
+    O = torch.zeros_like(Q)
+    act, n_act = i32([0, 1, 2, 3]), i32([4])
+    with pytest.raises(fc.FcError, match="workspace"):
+        ctx.chunk_decide(Q.view(-1), K.view(-1)[:Q.numel()], [0, Q.numel()], i32([0]), 1, 0.1,
+                         torch.zeros(1, device="cuda"), ws=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(fc.FcError, match="unsupported"):
+        ctx.chunk_attention(Q[:, :, :48].contiguous(), K[:, :, :48].contiguous(), V[:, :, :48].contiguous(),
+                            q_off, vis, slo, spo, act, n_act, O[:, :, :48].contiguous())
+    with pytest.raises(fc.FcError, match="aligned"):
+        Qm = torch.zeros(Q.numel() + 4, device="cuda")[1:1 + Q.numel()].view_as(Q)  # base off by 4 bytes
+        ctx.chunk_attention(Qm, K, V, q_off, vis, slo, spo, act, n_act, O)
+    with pytest.raises(fc.FcError, match="invalid"):
+        ctx.kv_score(Q[:, :50], K, pool_k=4)
+    with pytest.raises(fc.FcError, match="invalid"):
+        bad_vis = vis.copy()
+        bad_vis[-1] += 1  # beyond the logical length
+        ctx.chunk_attention(Q, K, V, q_off, bad_vis, slo, spo, act, n_act, O)
+    torch.cuda.synchronize()
+    assert (O == 0).all()

@@ -50,7 +50,8 @@ typedef enum {
   FC_ERR_WORKSPACE = -4,   /* ws is NULL or ws_bytes is below fc_*_workspace_bytes() */
   FC_ERR_DEVICE = -5,      /* the device is not compute capability 10.x */
   FC_ERR_CUDA = -6,        /* a CUDA runtime / driver call failed (see fc_last_cuda_error) */
-  FC_ERR_UNIMPLEMENTED = -7
+  FC_ERR_UNIMPLEMENTED = -7,
+  FC_ERR_TOO_LARGE = -8    /* the problem needs more scratch than a no-allocation entry point holds */
 } fc_status;
 
 typedef enum { FC_BF16 = 0, FC_F32 = 1 } fc_dtype;
@@ -109,6 +110,33 @@ int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const void* prev
                     int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
                     uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
                     uint32_t* status, void* ws, size_t ws_bytes);
+
+/* fc_chunk_decide_static — fc_chunk_decide without a workspace argument.
+ *
+ * The paper has no counterpart: this entry point exists for callers that may not allocate device
+ * memory at the point of the call — code running inside a memory-pool or allocator callback, a
+ * real-time loop that must not touch the allocator, a host that was handed fixed buffers by
+ * another runtime — and therefore have no workspace to pass.  The (num, den) slab pairs go to an
+ * array of fc_chunk_decide_static_max_bytes() = 1 MiB that is part of the library image: every
+ * GPU that loads the library holds it until the process exits.  Inputs, outputs and semantics are
+ * exactly those of fc_chunk_decide.
+ *
+ *   - Limit: fc_chunk_decide_workspace_bytes(total elements, n_chunks) must not exceed the
+ *     array, which holds 65,536 slab pairs: about 268 million elements over all chunks together,
+ *     whatever the dtype.  Beyond it the call returns FC_ERR_TOO_LARGE and launches nothing.
+ *   - The call never allocates or frees device memory.  The first call on each device looks up
+ *     the array's device address (a driver query, made with that device current); make that
+ *     first call before starting any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents.
+ *     Nothing in it has to start at zero (each slab pair is written before it is read), but two
+ *     calls that overlap on the GPU (different streams, no dependency) race on it: serialise
+ *     them, or use fc_chunk_decide with separate workspaces. */
+size_t fc_chunk_decide_static_max_bytes(void);
+int fc_chunk_decide_static(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
+                           const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
+                           int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
+                           uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
+                           uint32_t* status);
 
 /* ------------------------------------------------------------------------------------------
  * fc_chunk_attention — chunk-causal attention of the active chunks.

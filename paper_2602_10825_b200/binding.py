@@ -56,7 +56,7 @@ def lib():
         L = C.CDLL(_LIB_PATH)
         L.fc_status_string.restype = C.c_char_p
         L.fc_last_cuda_error.restype = C.c_char_p
-        for name in ("fc_chunk_decide_workspace_bytes", "fc_chunk_attention_workspace_bytes",
+        for name in ("fc_chunk_decide_static_max_bytes", "fc_chunk_decide_workspace_bytes", "fc_chunk_attention_workspace_bytes",
                      "fc_kv_score_workspace_bytes", "fc_kv_select_compact_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.fc_chunk_decide_workspace_bytes.argtypes = [C.c_int64, C.c_int]
@@ -172,6 +172,23 @@ class Context:
             _dev(active_ids, "active_ids", torch.int32), _dev(n_active, "n_active", torch.int32),
             _dev(status, "status", torch.int32), _dev(ws, "ws"), C.c_size_t(ws.numel()))
         self._check(rc, "fc_chunk_decide")
+        return dict(l1rel=l1rel, recompute=recompute, active_ids=active_ids, n_active=n_active, acc=acc)
+
+    def chunk_decide_static(self, cur, prev, chunk_elem_off, chunk_step, warmup_m, eps, acc, *, l1rel, recompute,
+                            active_ids, n_active, force=None, status=None):
+        """fc_chunk_decide_static: the decision without a workspace, for callers that cannot allocate device
+        memory (the scratch is a fixed 1 MiB array inside the library).  Every output tensor is passed in, so
+        this wrapper allocates nothing on the device either."""
+        off = np.ascontiguousarray(np.asarray(chunk_elem_off, dtype=np.int64))
+        n = len(off) - 1
+        rc = self._L.fc_chunk_decide_static(
+            self._h, self._stream(), _dev(cur, "cur"), _dev(prev, "prev"), _dt(cur),
+            off.ctypes.data_as(C.c_void_p), n, _dev(chunk_step, "chunk_step", torch.int32), int(warmup_m),
+            C.c_float(eps), _dev(force, "force", torch.uint8), _dev(acc, "acc", torch.float32),
+            _dev(l1rel, "l1rel", torch.float32), _dev(recompute, "recompute", torch.uint8),
+            _dev(active_ids, "active_ids", torch.int32), _dev(n_active, "n_active", torch.int32),
+            _dev(status, "status", torch.int32))
+        self._check(rc, "fc_chunk_decide_static")
         return dict(l1rel=l1rel, recompute=recompute, active_ids=active_ids, n_active=n_active, acc=acc)
 
     # ------------------------------------------------------------------ fc_chunk_attention

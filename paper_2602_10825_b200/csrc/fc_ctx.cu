@@ -24,6 +24,7 @@ extern "C" const char* fc_status_string(int status) {
     case FC_ERR_DEVICE: return "device is not compute capability 10.x";
     case FC_ERR_CUDA: return "CUDA call failed";
     case FC_ERR_UNIMPLEMENTED: return "not implemented";
+    case FC_ERR_TOO_LARGE: return "problem exceeds the built-in scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }

@@ -209,3 +209,62 @@ extern "C" int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const
   FC_LAUNCH_CHECK("decide_finalize_kernel");
   return FC_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// fc_chunk_decide_static: the same decision for callers that cannot allocate device memory.
+//
+// The slab partials live in a fixed array inside the library image instead of a caller workspace.
+// In host code the array's name is only a handle; its device address is looked up once per
+// device, with that device current, and that address is what the kernels receive.
+namespace {
+
+constexpr size_t kStaticScratchBytes = 1u << 20;  // 65,536 slabs of 16 KiB per tensor
+static __device__ __align__(256) unsigned char g_decide_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_scratch_addr[kMaxDevices] = {};  // device address of g_decide_scratch on each device (0 = not looked up)
+
+// Look the address up on first use per device.  Not an allocation: the array is part of the
+// module image every device already holds.  Concurrent first calls may both do the lookup; they
+// get the same answer.
+int static_scratch(int device, void** out) {
+  if (device < 0 || device >= kMaxDevices) return FC_ERR_UNSUPPORTED;
+  if (!g_scratch_addr[device]) {
+    int current = -1;
+    FC_CUDA_CHECK(cudaGetDevice(&current));
+    if (current != device) FC_CUDA_CHECK(cudaSetDevice(device));
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_decide_scratch);
+    if (current != device) cudaSetDevice(current);
+    if (e != cudaSuccess || !p) {
+      fc::set_cuda_error(e, "cudaGetSymbolAddress(g_decide_scratch)");
+      return FC_ERR_CUDA;
+    }
+    g_scratch_addr[device] = p;
+  }
+  *out = g_scratch_addr[device];
+  return FC_OK;
+}
+
+}  // namespace
+
+extern "C" size_t fc_chunk_decide_static_max_bytes(void) { return kStaticScratchBytes; }
+
+extern "C" int fc_chunk_decide_static(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
+                                      const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
+                                      int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
+                                      uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
+                                      uint32_t* status) {
+  if (!ctx || !chunk_elem_off || n_chunks <= 0) return FC_ERR_INVALID_ARG;
+  if (n_chunks > FC_MAX_CHUNKS) return FC_ERR_UNSUPPORTED;
+  const int64_t total = chunk_elem_off[n_chunks];
+  if (total < 0) return FC_ERR_INVALID_ARG;
+  if (fc_chunk_decide_workspace_bytes(total, n_chunks) > kStaticScratchBytes) return FC_ERR_TOO_LARGE;
+  void* scratch = nullptr;
+  const int rc = static_scratch(ctx->device, &scratch);
+  if (rc != FC_OK) return rc;
+  // Every slab pair is written by the reduction before the finalising kernel reads it, so the
+  // array needs no clearing between calls even though it keeps the previous call's contents.
+  return fc_chunk_decide(ctx, stream, cur, prev, dtype, chunk_elem_off, n_chunks, chunk_step, warmup_m, eps, force,
+                         acc, l1rel, recompute, active_ids, n_active, status, scratch, kStaticScratchBytes);
+}

@@ -1,6 +1,8 @@
 // Geometry shared by the two attention kernels of libfc (CUDA-core and tcgen05).
 #pragma once
 
+#include <cuda.h>
+
 #include "fc_common.cuh"
 
 namespace fc {
@@ -26,6 +28,9 @@ int attention_simt(cudaStream_t st, const AttnGeom& g, const void* Q, const void
 int attention_tc(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const void* Q, const void* K,
                  const void* V, void* O, void* ws, size_t ws_bytes);
 size_t attention_tc_workspace_bytes();
+// warp-specialised kernel; tensor maps as built by attention_tc
+int attention_ws_launch(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const CUtensorMap& tq,
+                        const CUtensorMap& tk, const CUtensorMap& tv, void* O);
 bool attention_tc_supported(const AttnGeom& g, int dtype);
 
 }  // namespace fc

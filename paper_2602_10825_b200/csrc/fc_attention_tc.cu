@@ -11,6 +11,7 @@
 // Every mbarrier wait is bounded; a wait that gives up sets FC_DEV_TIMEOUT and the kernel runs on
 // to its normal teardown (tensor memory is always released).
 #include <cmath>
+#include <cstdlib>
 
 #include "fc_attention.cuh"
 #include "fc_tcgen05.cuh"
@@ -322,6 +323,7 @@ int attention_tc(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g_in, const void*
   if ((rc = make_tmap(ctx, &tq, Q, g.d, q_rows, g.H_q, g.q_rs, g.H_q > 1 ? g.q_hs : g.q_rs * q_rows)) != FC_OK) return rc;
   if ((rc = make_tmap(ctx, &tk, K, g.d, g.kv_rows, g.H_kv, g.k_rs, g.H_kv > 1 ? g.k_hs : g.k_rs * g.kv_rows)) != FC_OK) return rc;
   if ((rc = make_tmap(ctx, &tv, V, g.d, g.kv_rows, g.H_kv, g.v_rs, g.H_kv > 1 ? g.v_hs : g.v_rs * g.kv_rows)) != FC_OK) return rc;
+  if (!getenv("FC_ATTN_BASIC")) return attention_ws_launch(ctx, st, g, tq, tk, tv, O);
   uint32_t* counter = (uint32_t*)ws;
   FC_CUDA_CHECK(cudaMemsetAsync(counter, 0, sizeof(uint32_t), st));
   const int64_t items = (int64_t)max_tiles * g.H_q;

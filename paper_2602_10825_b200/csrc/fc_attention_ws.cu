@@ -1,0 +1,397 @@
+// Chunk-causal attention on tcgen05 tensor cores, warp-specialised (bf16 in, fp32 accumulation).
+//
+// One persistent CTA per SM (384 threads, all 512 tensor-memory columns).  A work item is
+// (head, active chunk, pair of 128-row query tiles A and B); items are ordered head-major with the
+// longest visible prefix first and dealt round-robin to the CTAs.  Roles:
+//   warps 0-3  softmax of tile A     one query row per thread, online softmax in the exp2 domain
+//   warps 4-7  softmax of tile B
+//   warp  8    TMA producer          Q pair once per item, then K and V tiles into 2-stage rings
+//   warp  9    MMA issuer            S_A(j), PV_B(j-1), S_B(j), PV_A(j), ... so the tensor pipe
+//                                    always has the other tile's work while one tile is in softmax
+// Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512); P (bf16) overwrites the
+// low half of its S.  tcgen05.mma executes in issue order, so S_X(j+1) cannot overtake PV_X(j),
+// which still reads P_X(j), and "S_X(j) is complete" implies "PV_X(j-1) is complete", which is
+// what lets the softmax warps rescale O_X in place when a row maximum moves.
+// The rescale is lazy: a row keeps its reference maximum until the true maximum exceeds it by more
+// than 2^8, so P stays below 256 and O is rescaled only a few times per row.
+// Every mbarrier wait is bounded (see mbar_wait_bounded); tensor memory is always released.
+#include <cmath>
+
+#include "fc_attention.cuh"
+#include "fc_tcgen05.cuh"
+#include "fc_tcgen05_ld.cuh"
+
+namespace {
+
+using namespace fc::sm100;
+
+constexpr int kBM = 128, kBN = 128;
+constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {TMA warp, MMA warp, 2 spare warps}
+constexpr int kStages = 2;
+constexpr uint32_t kTmemCols = 512;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
+
+struct WsSmem {
+  uint64_t q_full, q_empty;
+  uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  uint64_t s_full[2], p_ready[2], o_done[2];
+  uint32_t tmem_base;
+  uint32_t abort;
+  int32_t n_act, tiles_per_head;
+  int32_t act_chunk[FC_MAX_CHUNKS];
+  int32_t act_item_end[FC_MAX_CHUNKS];  // running item (tile-pair) count over the descending active list
+};
+
+struct Item {
+  int h, hk, c, row0, n_vis;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                    const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ fc::AttnGeom g,
+                    __nv_bfloat16* __restrict__ O) {
+  constexpr uint32_t kTileBytes = kBM * D * 2;
+  constexpr int kAtoms = D / 64;
+  constexpr uint32_t kAtomBytes = kBM * 128;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t q_s = smem_u32(smem);                 // Q_A, Q_B
+  const uint32_t k_s = q_s + 2 * kTileBytes;           // K ring
+  const uint32_t v_s = k_s + kStages * kTileBytes;     // V ring
+  WsSmem* sh = (WsSmem*)(smem + (2 + 2 * kStages) * kTileBytes);
+  volatile uint32_t* abort = &sh->abort;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    mbar_init(smem_u32(&sh->q_full), 1);
+    mbar_init(smem_u32(&sh->q_empty), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&sh->k_full[s]), 1);
+      mbar_init(smem_u32(&sh->k_empty[s]), 1);
+      mbar_init(smem_u32(&sh->v_full[s]), 1);
+      mbar_init(smem_u32(&sh->v_empty[s]), 1);
+    }
+    for (int x = 0; x < 2; ++x) {
+      mbar_init(smem_u32(&sh->s_full[x]), 1);
+      mbar_init(smem_u32(&sh->p_ready[x]), 4);  // one arrival per softmax warp
+      mbar_init(smem_u32(&sh->o_done[x]), 1);
+    }
+    mbar_fence_init();
+    sh->abort = 0;
+    tma_prefetch_desc(&tmap_q);
+    tma_prefetch_desc(&tmap_k);
+    tma_prefetch_desc(&tmap_v);
+    const int n_in = min(max(*g.n_active, 0), g.W);
+    int n = 0, items = 0;
+    for (int a = n_in - 1; a >= 0; --a) {
+      const int c = g.active_ids[a];
+      if (c < 0 || c >= g.W) {
+        if (g.status) atomicOr(g.status, FC_DEV_BAD_INDEX);
+        continue;
+      }
+      items += (g.q_row_off[c + 1] - g.q_row_off[c] + 2 * kBM - 1) / (2 * kBM);
+      sh->act_chunk[n] = c;
+      sh->act_item_end[n] = items;
+      ++n;
+    }
+    sh->n_act = n;
+    sh->tiles_per_head = items;
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&sh->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh->tmem_base;
+  const int n_act = sh->n_act, per_head = sh->tiles_per_head;
+  const int total_items = per_head * g.H_q;
+
+  auto decode = [&](int item) {
+    Item it;
+    it.h = item / per_head;
+    const int rem = item % per_head;
+    int a = 0;
+    while (a + 1 < n_act && rem >= sh->act_item_end[a]) ++a;
+    it.c = sh->act_chunk[a];
+    it.row0 = g.q_row_off[it.c] + (rem - (a > 0 ? sh->act_item_end[a - 1] : 0)) * 2 * kBM;
+    it.n_vis = g.vis[it.c];
+    it.hk = it.h / g.group;
+    return it;
+  };
+
+  auto count_tiles = [&](const Item& it) {
+    int n = 0;
+    for (int s = 0; s < g.n_seg; ++s) {
+      const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
+      if (seg_vis <= 0) break;
+      n += (seg_vis + kBN - 1) / kBN;
+    }
+    return n;
+  };
+
+  // Registers move from the third warpgroup, which only issues copies and MMAs, to the softmax
+  // warpgroups, which hold a 128-column row of S per thread: 256 x 224 + 128 x 56 <= 64 Ki.
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  if (warp == 8) {
+    // ------------------------------------------------------------------ TMA producer
+    uint32_t kv = 0, it_n = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++it_n) {
+      const Item it = decode(item);
+      mbar_wait_bounded(smem_u32(&sh->q_empty), (it_n & 1) ^ 1, abort);
+      if (lane == 0) {
+        mbar_expect_tx(smem_u32(&sh->q_full), 2 * kTileBytes);
+        for (int t = 0; t < 2; ++t)
+          for (int x = 0; x < kAtoms; ++x)
+            tma_load_3d(q_s + t * kTileBytes + x * kAtomBytes, &tmap_q, smem_u32(&sh->q_full), x * 64,
+                        it.row0 + t * kBM, it.h);
+      }
+      for (int s = 0; s < g.n_seg; ++s) {
+        const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
+        if (seg_vis <= 0) break;
+        for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv) {
+          const int st = kv % kStages, ph = (kv / kStages) & 1, prow = g.seg_phys[s] + j0;
+          mbar_wait_bounded(smem_u32(&sh->k_empty[st]), ph ^ 1, abort);
+          if (lane == 0) {
+            mbar_expect_tx(smem_u32(&sh->k_full[st]), kTileBytes);
+            for (int x = 0; x < kAtoms; ++x)
+              tma_load_3d(k_s + st * kTileBytes + x * kAtomBytes, &tmap_k, smem_u32(&sh->k_full[st]), x * 64, prow,
+                          it.hk);
+          }
+          mbar_wait_bounded(smem_u32(&sh->v_empty[st]), ph ^ 1, abort);
+          if (lane == 0) {
+            mbar_expect_tx(smem_u32(&sh->v_full[st]), kTileBytes);
+            for (int x = 0; x < kAtoms; ++x)
+              tma_load_3d(v_s + st * kTileBytes + x * kAtomBytes, &tmap_v, smem_u32(&sh->v_full[st]), x * 64, prow,
+                          it.hk);
+          }
+          __syncwarp();
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------------------------------------------ MMA issuer
+    constexpr uint32_t kIdescQK = idesc_bf16_f32(kBM, kBN, false, false);
+    constexpr uint32_t kIdescPV = idesc_bf16_f32(kBM, D, false, true);
+    auto issue_s = [&](int x, int st) {  // S_x = Q_x K^T
+#pragma unroll
+      for (int kk = 0; kk < D / 16; ++kk) {
+        const uint32_t off = (kk / 4) * kAtomBytes + (kk % 4) * 32;
+        umma_ss(tmem + x * 128, smem_desc_sw128(q_s + x * kTileBytes + off, 16, 1024),
+                smem_desc_sw128(k_s + st * kTileBytes + off, 16, 1024), kIdescQK, kk > 0);
+      }
+    };
+    auto issue_pv = [&](int x, int st, bool accumulate) {  // O_x (+)= P_x V
+#pragma unroll
+      for (int kk = 0; kk < kBN / 16; ++kk)
+        umma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8,
+                smem_desc_sw128(v_s + st * kTileBytes + kk * 2048, kAtomBytes, 1024), kIdescPV, accumulate || kk > 0);
+    };
+    uint32_t kv = 0, it_n = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++it_n) {
+      const Item it = decode(item);
+      const int n_tiles = count_tiles(it);
+      mbar_wait_bounded(smem_u32(&sh->q_full), it_n & 1, abort);
+      tc_fence_after();
+      if (n_tiles == 0 && lane == 0) umma_commit(smem_u32(&sh->q_empty));
+      int j = 0;  // tile index inside the item
+      for (int s = 0; s < g.n_seg; ++s) {
+        const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
+        if (seg_vis <= 0) break;
+        for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv, ++j) {
+          const int st = kv % kStages, ph = (kv / kStages) & 1;
+          mbar_wait_bounded(smem_u32(&sh->k_full[st]), ph, abort);
+          tc_fence_after();
+          if (lane == 0) {
+            issue_s(0, st);
+            umma_commit(smem_u32(&sh->s_full[0]));
+          }
+          if (j > 0) {  // PV_B of the previous tile
+            const uint32_t pkv = kv - 1;
+            mbar_wait_bounded(smem_u32(&sh->p_ready[1]), pkv & 1, abort);
+            tc_fence_after();
+            if (lane == 0) {
+              issue_pv(1, pkv % kStages, j > 1);
+              umma_commit(smem_u32(&sh->v_empty[pkv % kStages]));
+            }
+          }
+          if (lane == 0) {
+            issue_s(1, st);
+            umma_commit(smem_u32(&sh->s_full[1]));
+            umma_commit(smem_u32(&sh->k_empty[st]));
+            if (j == n_tiles - 1) umma_commit(smem_u32(&sh->q_empty));  // last read of the Q pair
+          }
+          mbar_wait_bounded(smem_u32(&sh->p_ready[0]), kv & 1, abort);
+          mbar_wait_bounded(smem_u32(&sh->v_full[st]), ph, abort);
+          tc_fence_after();
+          if (lane == 0) issue_pv(0, st, j > 0);
+          __syncwarp();
+        }
+      }
+      if (j > 0) {
+        const uint32_t pkv = kv - 1;
+        mbar_wait_bounded(smem_u32(&sh->p_ready[1]), pkv & 1, abort);
+        tc_fence_after();
+        if (lane == 0) {
+          issue_pv(1, pkv % kStages, j > 1);
+          umma_commit(smem_u32(&sh->v_empty[pkv % kStages]));
+        }
+      }
+      if (lane == 0) {
+        umma_commit(smem_u32(&sh->o_done[0]));
+        umma_commit(smem_u32(&sh->o_done[1]));
+      }
+      __syncwarp();
+    }
+  }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    // ------------------------------------------------------------------ softmax + epilogue, tile x
+    const int x = warp >> 2;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t t_s = tmem + lane_base + x * 128;
+    const uint32_t t_o = tmem + lane_base + 256 + x * 128;
+    const int r_in = (warp & 3) * 32 + lane;  // row inside the tile
+    const float scale_log2 = g.scale * 1.4426950408889634f;
+    uint32_t kv = 0, it_n = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++it_n) {
+      const Item it = decode(item);
+      float m = -INFINITY, l = 0.f;
+      int j = 0;
+      for (int s = 0; s < g.n_seg; ++s) {
+        const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
+        if (seg_vis <= 0) break;
+        for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv, ++j) {
+          const int cols_valid = min(kBN, seg_vis - j0);
+          mbar_wait_bounded(smem_u32(&sh->s_full[x]), kv & 1, abort);
+          tc_fence_after();
+          uint32_t sv[kBN];
+          tmem_ld128_wait(t_s, sv);
+          float tile_max = -INFINITY;
+          if (cols_valid == kBN) {
+#pragma unroll
+            for (int i = 0; i < kBN; ++i) tile_max = fmaxf(tile_max, __uint_as_float(sv[i]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < kBN; ++i) {
+              if (i >= cols_valid) sv[i] = 0xff800000u;  // -inf
+              tile_max = fmaxf(tile_max, __uint_as_float(sv[i]));
+            }
+          }
+          tile_max *= scale_log2;  // scale > 0
+          // lazy reference update: move only when the maximum grew by more than the threshold
+          float alpha = 1.f;
+          const bool move = tile_max > m + kRescaleThreshold;  // always true on the first tile (m = -inf)
+          if (move) {
+            alpha = ex2(m - tile_max);
+            m = tile_max;
+          }
+          if (j > 0 && __any_sync(0xffffffffu, move)) {
+#pragma unroll
+            for (int q4 = 0; q4 < D / 32; ++q4) {
+              uint32_t r[32];
+              tmem_ld32_wait(t_o + q4 * 32, r);
+#pragma unroll
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+              tmem_st32(t_o + q4 * 32, r);
+            }
+          }
+          float row_sum = 0.f;
+          const float neg_m = -m;
+#pragma unroll
+          for (int q2 = 0; q2 < kBN / 32; ++q2) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float p0 = ex2(fmaf(__uint_as_float(sv[q2 * 32 + 2 * i]), scale_log2, neg_m));
+              const float p1 = ex2(fmaf(__uint_as_float(sv[q2 * 32 + 2 * i + 1]), scale_log2, neg_m));
+              row_sum += p0 + p1;
+              __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+              pk[i] = *reinterpret_cast<uint32_t*>(&b);
+            }
+            tmem_st16(t_s + q2 * 16, pk);
+          }
+          l = l * alpha + row_sum;
+          tmem_wait_st();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready[x]));
+        }
+      }
+      // epilogue
+      mbar_wait_bounded(smem_u32(&sh->o_done[x]), it_n & 1, abort);
+      tc_fence_after();
+      const int row = it.row0 + x * kBM + r_in;
+      const bool row_ok = row < g.q_row_off[it.c + 1];
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+      __nv_bfloat16* out = O + (int64_t)it.h * g.o_hs + (int64_t)row * g.o_rs;
+#pragma unroll
+      for (int q4 = 0; q4 < D / 32; ++q4) {
+        uint32_t r[32];
+        if (j > 0) {
+          tmem_ld32_wait(t_o + q4 * 32, r);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = 0;
+        }
+        if (row_ok) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 w;
+            uint32_t* wp = &w.x;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2 * i]) * inv,
+                                                       __uint_as_float(r[v * 8 + 2 * i + 1]) * inv);
+              wp[i] = *reinterpret_cast<uint32_t*>(&b);
+            }
+            *reinterpret_cast<uint4*>(out + q4 * 32 + v * 8) = w;
+          }
+        }
+      }
+      if (g.lse && row_ok)
+        g.lse[(int64_t)it.h * g.lse_hs + row] = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+      tc_fence_before();  // O_x has been read before this warp's next p_ready arrival lets PV_x overwrite it
+    }
+  }
+
+  if (*abort) {
+    // something never arrived: give copies and instructions still in flight time to land before the
+    // shared and tensor memory of this CTA are handed back
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *abort && g.status) atomicOr(g.status, FC_DEV_TIMEOUT);
+  if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+}
+
+}  // namespace
+
+namespace fc {
+
+int attention_ws_launch(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const CUtensorMap& tq,
+                        const CUtensorMap& tk, const CUtensorMap& tv, void* O) {
+  int max_items = 0;
+  for (int c = 0; c < g.W; ++c) max_items += (g.q_row_off[c + 1] - g.q_row_off[c] + 2 * kBM - 1) / (2 * kBM);
+  const int64_t items = (int64_t)max_items * g.H_q;
+  if (items == 0) return FC_OK;
+  const int grid = (int)std::min<int64_t>(items, (int64_t)ctx->sm_count);
+  // at least half of the shared memory, so that a second CTA (and its 512 columns) never joins the SM
+  const size_t need = (2 + 2 * kStages) * (size_t)kBM * g.d * 2 + sizeof(WsSmem) + 1024;
+  const size_t smem = std::max<size_t>(need, 120 * 1024);
+  if (g.d == 128) {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(attention_ws_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attention_ws_kernel<128><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O);
+  } else {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(attention_ws_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    attention_ws_kernel<64><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O);
+  }
+  FC_LAUNCH_CHECK("attention_ws_kernel");
+  return FC_OK;
+}
+
+}  // namespace fc

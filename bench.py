@@ -56,7 +56,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.t = threading.Thread(target=self._read, daemon=True)
             self.t.start()
         except OSError:
@@ -227,9 +227,9 @@ def oracle_sample(w, seed, n_rows):
     import oracle
     Q, K, V = wl.qkv(w, seed)
     q_off, vis, slo, spo = wl.prefix_layout(w)
-    rows = wl.sample_rows(w, 0, seed)
-    pick = np.linspace(0, len(rows) - 1, n_rows).astype(int)
-    rows = rows[pick]
+    rows = wl.sample_rows(w, n_rows, seed)
+    if len(rows) > n_rows:
+        rows = rows[np.unique(np.linspace(0, len(rows) - 1, n_rows).astype(int))]
     Qb, Kb, Vb = wl.bits(Q), wl.bits(K), wl.bits(V)
     cores = oracle.hardware_threads()
     t = time.perf_counter()
@@ -246,7 +246,7 @@ def run_reference(args, w):
     import oracle
     oracle.build()
     times, flops = [], 0.0
-    n_rows = 4
+    n_rows = 48
     for k in range(args.warmup + args.steps):
         dt, fl, cores, desc = oracle_sample(w, k, n_rows)
         if k >= args.warmup:
@@ -269,8 +269,8 @@ def run_reference(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--config", default="single_step_bf16", choices=sorted(wl.CONFIGS))
     ap.add_argument("--impl", default="fc", choices=["fc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -319,8 +319,8 @@ def main():
 
     e2e = None
     if not args.no_e2e:
-        e2e_ms, h2d, d2h = time_e2e(step, max(2, args.steps // 4), args.warmup, barrier)
-        e2e_steps = max(2, args.steps // 4)
+        e2e_steps = max(2, min(args.steps // 4, 40))
+        e2e_ms, h2d, d2h = time_e2e(step, e2e_steps, args.warmup, barrier)
     if dist is not None:
         t = torch.tensor([total_ms, e2e_ms / e2e_steps if not args.no_e2e else 0.0], device=device, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -347,7 +347,7 @@ def main():
                        "parallelism": "replicas" if world > 1 else "single"},
             "stages_ms": stage_ms,
             "roofline": {"bound": "tensor", "achieved": attn_tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": attn_tflops / peaks["bf16_tflops"], "traffic": None, "kernel": "attention_tc_kernel",
+                         "frac": attn_tflops / peaks["bf16_tflops"], "traffic": None, "kernel": "attention_ws_kernel",
                          "peak_kind": peak_kind + " burst", "frac_of_nominal": attn_tflops / NOMINAL["bf16_tflops"],
                          "frac_of_sustained": attn_tflops / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])},
             "roofline_compact": {"bound": "hbm", "achieved": compact_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -363,7 +363,7 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
-            dt, fl, cores, desc = oracle_sample(w, 0, 8)
+            dt, fl, cores, desc = oracle_sample(w, 0, 768)
             line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                     "sample": desc + f" ({dt:.1f} s)"}
         print(json.dumps(line))

@@ -159,7 +159,8 @@ typedef struct {
   int64_t o_hs, o_rs;
   int64_t kv_rows;                           /* physical rows per head in the K/V store */
   float scale;                               /* 0 => 1/sqrt(d) */
-  int32_t impl;                              /* 0 auto; 1 force the CUDA-core kernel; 2 force tcgen05 */
+  int32_t impl;                              /* 0 auto; 1 force the CUDA-core kernel; 2 force tcgen05
+                                                (warp-specialised); 3 force the single-stage tcgen05 kernel */
 } fc_attn_desc;
 
 /*   Q, O             DEVICE [H_q, rows, d]; K, V DEVICE [H_kv, kv_rows, d]; `dtype` elements.

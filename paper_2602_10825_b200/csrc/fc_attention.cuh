@@ -25,12 +25,14 @@ struct AttnGeom {
 int attention_simt(cudaStream_t st, const AttnGeom& g, const void* Q, const void* K, const void* V,
                    int dtype, void* O);
 // bf16 only, segment-table addressing only.
+// `basic` selects the single-stage kernel (one CTA per tile, no warp roles) instead of the
+// warp-specialised one.
 int attention_tc(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const void* Q, const void* K,
-                 const void* V, void* O, void* ws, size_t ws_bytes);
+                 const void* V, void* O, void* ws, size_t ws_bytes, bool basic);
 size_t attention_tc_workspace_bytes();
-// warp-specialised kernel; tensor maps as built by attention_tc
+// warp-specialised kernel; tensor maps as built by attention_tc, `counter` = 4 bytes of workspace
 int attention_ws_launch(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const CUtensorMap& tq,
-                        const CUtensorMap& tk, const CUtensorMap& tv, void* O);
+                        const CUtensorMap& tk, const CUtensorMap& tv, void* O, uint32_t* counter);
 bool attention_tc_supported(const AttnGeom& g, int dtype);
 
 }  // namespace fc

@@ -11,7 +11,6 @@
 // Every mbarrier wait is bounded; a wait that gives up sets FC_DEV_TIMEOUT and the kernel runs on
 // to its normal teardown (tensor memory is always released).
 #include <cmath>
-#include <cstdlib>
 
 #include "fc_attention.cuh"
 #include "fc_tcgen05.cuh"
@@ -295,7 +294,7 @@ bool attention_tc_supported(const AttnGeom& g, int dtype) {
 }
 
 int attention_tc(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g_in, const void* Q, const void* K, const void* V,
-                 void* O, void* ws, size_t ws_bytes) {
+                 void* O, void* ws, size_t ws_bytes, bool basic) {
   if (!ws || ws_bytes < attention_tc_workspace_bytes()) return FC_ERR_WORKSPACE;
   if (!aligned16(ws)) return FC_ERR_MISALIGNED;
   AttnGeom g = g_in;
@@ -323,8 +322,8 @@ int attention_tc(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g_in, const void*
   if ((rc = make_tmap(ctx, &tq, Q, g.d, q_rows, g.H_q, g.q_rs, g.H_q > 1 ? g.q_hs : g.q_rs * q_rows)) != FC_OK) return rc;
   if ((rc = make_tmap(ctx, &tk, K, g.d, g.kv_rows, g.H_kv, g.k_rs, g.H_kv > 1 ? g.k_hs : g.k_rs * g.kv_rows)) != FC_OK) return rc;
   if ((rc = make_tmap(ctx, &tv, V, g.d, g.kv_rows, g.H_kv, g.v_rs, g.H_kv > 1 ? g.v_hs : g.v_rs * g.kv_rows)) != FC_OK) return rc;
-  if (!getenv("FC_ATTN_BASIC")) return attention_ws_launch(ctx, st, g, tq, tk, tv, O);
   uint32_t* counter = (uint32_t*)ws;
+  if (!basic) return attention_ws_launch(ctx, st, g, tq, tk, tv, O, counter);
   FC_CUDA_CHECK(cudaMemsetAsync(counter, 0, sizeof(uint32_t), st));
   const int64_t items = (int64_t)max_tiles * g.H_q;
   const int grid = (int)std::min<int64_t>(items, 2 * (int64_t)ctx->sm_count);

@@ -1,11 +1,14 @@
 // Chunk-causal attention on tcgen05 tensor cores, warp-specialised (bf16 in, fp32 accumulation).
 //
 // One persistent CTA per SM (384 threads, all 512 tensor-memory columns).  A work item is
-// (head, active chunk, pair of 128-row query tiles A and B); items are ordered head-major with the
-// longest visible prefix first and dealt round-robin to the CTAs.  Roles:
+// (active chunk, head, pair of 128-row query tiles A and B).  Items are ordered by the length of
+// the chunk's visible prefix, longest first, and handed out through a device counter, so the
+// last items to start are the shortest ones and the SMs finish together.  Roles:
 //   warps 0-3  softmax of tile A     one query row per thread, online softmax in the exp2 domain
 //   warps 4-7  softmax of tile B
-//   warp  8    TMA producer          Q pair once per item, then K and V tiles into 2-stage rings
+//   warp  8    scheduler + TMA       takes the next item off the counter, publishes it to the
+//                                    other warps through a 2-slot ring, then loads the Q pair and
+//                                    streams K and V tiles into 2-stage rings
 //   warp  9    MMA issuer            S_A(j), PV_B(j-1), S_B(j), PV_A(j), ... so the tensor pipe
 //                                    always has the other tile's work while one tile is in softmax
 // Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512); P (bf16) overwrites the
@@ -14,6 +17,9 @@
 // what lets the softmax warps rescale O_X in place when a row maximum moves.
 // The rescale is lazy: a row keeps its reference maximum until the true maximum exceeds it by more
 // than 2^8, so P stays below 256 and O is rescaled only a few times per row.
+// The softmax is written for issue slots and for the special-function unit, which at d = 128 is as
+// busy as the tensor pipe: three-input max, two-wide fp32 fma / add, one bf16x2 convert per
+// pair, and a share of the exponentials evaluated as a cubic on the fma pipe instead of ex2.
 // Every mbarrier wait is bounded (see mbar_wait_bounded); tensor memory is always released.
 #include <cmath>
 
@@ -30,27 +36,119 @@ constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {TMA warp,
 constexpr int kStages = 2;
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
+// of every 32 columns, this many (the last ones) take the polynomial exponential
+#ifndef FC_ATTN_EMU_COLS
+#define FC_ATTN_EMU_COLS 8
+#endif
+constexpr int kEmuCols = FC_ATTN_EMU_COLS;
 
 struct WsSmem {
   uint64_t q_full, q_empty;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[2], p_ready[2], o_done[2];
+  uint64_t it_full[2], it_empty[2];
+  int32_t it_slot[2];
   uint32_t tmem_base;
   uint32_t abort;
-  int32_t n_act, tiles_per_head;
-  int32_t act_chunk[FC_MAX_CHUNKS];
-  int32_t act_item_end[FC_MAX_CHUNKS];  // running item (tile-pair) count over the descending active list
+  int32_t n_act, total_items;
+  int32_t act_chunk[FC_MAX_CHUNKS];     // active chunks, longest visible prefix first
+  int32_t act_item_end[FC_MAX_CHUNKS];  // running item count over that list (all heads)
 };
 
 struct Item {
   int h, hk, c, row0, n_vis;
 };
 
+// ---- two-wide fp32 arithmetic and friends ------------------------------------------------------
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// {lo, hi} -> packed bf16 pair, lo in the low half
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+// 2^x for a pair, x <= 8, on the fma pipe: n = round(x) through the 1.5 * 2^23 shift, 2^(x-n) as a cubic
+// on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16 rounding of P), then n added to the exponent
+// field.  Inputs below -126 are clamped; their result is a harmless ~1e-38.
+__device__ __forceinline__ void ex2_poly2(float x0, float x1, float& y0, float& y1) {
+  const uint64_t kShift = pack2(12582912.f, 12582912.f), kUnshift = pack2(-12582912.f, -12582912.f);
+  const uint64_t kMinus1 = pack2(-1.f, -1.f);
+  const uint64_t c0 = pack2(0.9999280572f, 0.9999280572f), c1 = pack2(0.6932609677f, 0.6932609677f);
+  const uint64_t c2 = pack2(0.2426111251f, 0.2426111251f), c3 = pack2(0.0551716685f, 0.0551716685f);
+  const uint64_t x = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t t = add2(x, kShift);
+  const uint64_t n = add2(t, kUnshift);
+  const uint64_t f = fma2(n, kMinus1, x);
+  uint64_t p = fma2(c3, f, c2);
+  p = fma2(p, f, c1);
+  p = fma2(p, f, c0);
+  float p0, p1, t0, t1;
+  unpack2(p, p0, p1);
+  unpack2(t, t0, t1);
+  y0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+  y1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+}
+
+// P = 2^(S * scale - m) for one row of a 128-column tile, written back over S as bf16; returns the row sum.
+template <bool kAllEx2>
+__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s) {
+  const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
+  uint64_t sum2[2] = {0ull, 0ull};
+  constexpr int kEmuPairs = kAllEx2 ? 0 : kEmuCols / 2;
+#pragma unroll
+  for (int q2 = 0; q2 < kBN / 32; ++q2) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint64_t x = fma2(pack2(__uint_as_float(sv[q2 * 32 + 2 * i]), __uint_as_float(sv[q2 * 32 + 2 * i + 1])),
+                              sc2, nm2);
+      float x0, x1, p0, p1;
+      unpack2(x, x0, x1);
+      if (i >= 16 - kEmuPairs) {
+        ex2_poly2(x0, x1, p0, p1);
+      } else {
+        p0 = ex2(x0);
+        p1 = ex2(x1);
+      }
+      sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
+      pk[i] = cvt_bf16x2(p0, p1);
+    }
+    tmem_st16(t_s + q2 * 16, pk);
+  }
+  float a, b, c, d;
+  unpack2(sum2[0], a, b);
+  unpack2(sum2[1], c, d);
+  return (a + b) + (c + d);
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ fc::AttnGeom g,
-                    __nv_bfloat16* __restrict__ O) {
+                    __nv_bfloat16* __restrict__ O, uint32_t* __restrict__ counter) {
   constexpr uint32_t kTileBytes = kBM * D * 2;
   constexpr int kAtoms = D / 64;
   constexpr uint32_t kAtomBytes = kBM * 128;
@@ -76,27 +174,39 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       mbar_init(smem_u32(&sh->s_full[x]), 1);
       mbar_init(smem_u32(&sh->p_ready[x]), 4);  // one arrival per softmax warp
       mbar_init(smem_u32(&sh->o_done[x]), 1);
+      mbar_init(smem_u32(&sh->it_full[x]), 1);
+      mbar_init(smem_u32(&sh->it_empty[x]), 9);  // the MMA warp and the eight softmax warps
+      sh->it_slot[x] = -1;
     }
     mbar_fence_init();
     sh->abort = 0;
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
+    // active chunks sorted by visible length, longest first (insertion sort, at most 64 entries)
     const int n_in = min(max(*g.n_active, 0), g.W);
-    int n = 0, items = 0;
-    for (int a = n_in - 1; a >= 0; --a) {
+    int n = 0;
+    for (int a = 0; a < n_in; ++a) {
       const int c = g.active_ids[a];
       if (c < 0 || c >= g.W) {
         if (g.status) atomicOr(g.status, FC_DEV_BAD_INDEX);
         continue;
       }
-      items += (g.q_row_off[c + 1] - g.q_row_off[c] + 2 * kBM - 1) / (2 * kBM);
-      sh->act_chunk[n] = c;
-      sh->act_item_end[n] = items;
-      ++n;
+      int p = n++;
+      while (p > 0 && g.vis[sh->act_chunk[p - 1]] < g.vis[c]) {
+        sh->act_chunk[p] = sh->act_chunk[p - 1];
+        --p;
+      }
+      sh->act_chunk[p] = c;
+    }
+    int items = 0;
+    for (int a = 0; a < n; ++a) {
+      const int c = sh->act_chunk[a];
+      items += g.H_q * ((g.q_row_off[c + 1] - g.q_row_off[c] + 2 * kBM - 1) / (2 * kBM));
+      sh->act_item_end[a] = items;
     }
     sh->n_act = n;
-    sh->tiles_per_head = items;
+    sh->total_items = items;
   }
   if (warp == 0) {
     tmem_alloc(smem_u32(&sh->tmem_base), kTmemCols);
@@ -106,20 +216,31 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sh->tmem_base;
-  const int n_act = sh->n_act, per_head = sh->tiles_per_head;
-  const int total_items = per_head * g.H_q;
+  const int n_act = sh->n_act;
+  const int total_items = sh->total_items;
 
   auto decode = [&](int item) {
     Item it;
-    it.h = item / per_head;
-    const int rem = item % per_head;
     int a = 0;
-    while (a + 1 < n_act && rem >= sh->act_item_end[a]) ++a;
+    while (a + 1 < n_act && item >= sh->act_item_end[a]) ++a;
+    const int start = a > 0 ? sh->act_item_end[a - 1] : 0;
+    const int pairs = (sh->act_item_end[a] - start) / g.H_q;
     it.c = sh->act_chunk[a];
-    it.row0 = g.q_row_off[it.c] + (rem - (a > 0 ? sh->act_item_end[a - 1] : 0)) * 2 * kBM;
+    it.h = (item - start) / pairs;
+    it.row0 = g.q_row_off[it.c] + ((item - start) % pairs) * 2 * kBM;
     it.n_vis = g.vis[it.c];
     it.hk = it.h / g.group;
     return it;
+  };
+  // consumer side of the item ring; -1 once the list is exhausted or the CTA has given up
+  auto next_item = [&](uint32_t n) {
+    const int slot = n & 1;
+    mbar_wait_bounded(smem_u32(&sh->it_full[slot]), (n >> 1) & 1, abort);
+    int item = sh->it_slot[slot];
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&sh->it_empty[slot]));
+    if (*abort || item >= total_items) item = -1;
+    return item;
   };
 
   auto count_tiles = [&](const Item& it) {
@@ -137,9 +258,21 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   if (warp >= 8) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   if (warp == 8) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ scheduler + TMA producer
     uint32_t kv = 0, it_n = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++it_n) {
+    int next = 0;
+    if (lane == 0) next = (int)atomicAdd(counter, 1u);
+    while (true) {
+      int item = __shfl_sync(0xffffffffu, next, 0);
+      if (item >= total_items) item = -1;
+      const int slot = it_n & 1;
+      mbar_wait_bounded(smem_u32(&sh->it_empty[slot]), ((it_n >> 1) & 1) ^ 1, abort);
+      if (lane == 0) {
+        sh->it_slot[slot] = item < 0 ? total_items : item;
+        mbar_arrive(smem_u32(&sh->it_full[slot]));
+      }
+      if (item < 0 || *abort) break;
+      if (lane == 0) next = (int)atomicAdd(counter, 1u);  // in flight while this item's tiles are loaded
       const Item it = decode(item);
       mbar_wait_bounded(smem_u32(&sh->q_empty), (it_n & 1) ^ 1, abort);
       if (lane == 0) {
@@ -171,6 +304,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           __syncwarp();
         }
       }
+      ++it_n;
     }
   } else if (warp == 9) {
     // ------------------------------------------------------------------ MMA issuer
@@ -190,8 +324,10 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         umma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8,
                 smem_desc_sw128(v_s + st * kTileBytes + kk * 2048, kAtomBytes, 1024), kIdescPV, accumulate || kk > 0);
     };
-    uint32_t kv = 0, it_n = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++it_n) {
+    uint32_t kv = 0;
+    for (uint32_t it_n = 0;; ++it_n) {
+      const int item = next_item(it_n);
+      if (item < 0) break;
       const Item it = decode(item);
       const int n_tiles = count_tiles(it);
       mbar_wait_bounded(smem_u32(&sh->q_full), it_n & 1, abort);
@@ -256,8 +392,10 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const uint32_t t_o = tmem + lane_base + 256 + x * 128;
     const int r_in = (warp & 3) * 32 + lane;  // row inside the tile
     const float scale_log2 = g.scale * 1.4426950408889634f;
-    uint32_t kv = 0, it_n = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++it_n) {
+    uint32_t kv = 0;
+    for (uint32_t it_n = 0;; ++it_n) {
+      const int item = next_item(it_n);
+      if (item < 0) break;
       const Item it = decode(item);
       float m = -INFINITY, l = 0.f;
       int j = 0;
@@ -270,18 +408,19 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           tc_fence_after();
           uint32_t sv[kBN];
           tmem_ld128_wait(t_s, sv);
-          float tile_max = -INFINITY;
-          if (cols_valid == kBN) {
+          if (cols_valid < kBN) {
 #pragma unroll
-            for (int i = 0; i < kBN; ++i) tile_max = fmaxf(tile_max, __uint_as_float(sv[i]));
-          } else {
-#pragma unroll
-            for (int i = 0; i < kBN; ++i) {
+            for (int i = 0; i < kBN; ++i)
               if (i >= cols_valid) sv[i] = 0xff800000u;  // -inf
-              tile_max = fmaxf(tile_max, __uint_as_float(sv[i]));
-            }
           }
-          tile_max *= scale_log2;  // scale > 0
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int i = 0; i < kBN; i += 8) {
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4)
+              mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
+          }
+          const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
           // lazy reference update: move only when the maximum grew by more than the threshold
           float alpha = 1.f;
           const bool move = tile_max > m + kRescaleThreshold;  // always true on the first tile (m = -inf)
@@ -299,21 +438,9 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
               tmem_st32(t_o + q4 * 32, r);
             }
           }
-          float row_sum = 0.f;
-          const float neg_m = -m;
-#pragma unroll
-          for (int q2 = 0; q2 < kBN / 32; ++q2) {
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float p0 = ex2(fmaf(__uint_as_float(sv[q2 * 32 + 2 * i]), scale_log2, neg_m));
-              const float p1 = ex2(fmaf(__uint_as_float(sv[q2 * 32 + 2 * i + 1]), scale_log2, neg_m));
-              row_sum += p0 + p1;
-              __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-              pk[i] = *reinterpret_cast<uint32_t*>(&b);
-            }
-            tmem_st16(t_s + q2 * 16, pk);
-          }
+          // a ragged tile takes ex2 everywhere so that its masked columns give exactly 0
+          const float row_sum = cols_valid < kBN ? exp_tile<true>(sv, scale_log2, m, t_s)
+                                                 : exp_tile<false>(sv, scale_log2, m, t_s);
           l = l * alpha + row_sum;
           tmem_wait_st();
           tc_fence_before();
@@ -343,11 +470,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             uint4 w;
             uint32_t* wp = &w.x;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              __nv_bfloat162 b = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2 * i]) * inv,
-                                                       __uint_as_float(r[v * 8 + 2 * i + 1]) * inv);
-              wp[i] = *reinterpret_cast<uint32_t*>(&b);
-            }
+            for (int i = 0; i < 4; ++i)
+              wp[i] = cvt_bf16x2(__uint_as_float(r[v * 8 + 2 * i]) * inv, __uint_as_float(r[v * 8 + 2 * i + 1]) * inv);
             *reinterpret_cast<uint4*>(out + q4 * 32 + v * 8) = w;
           }
         }
@@ -374,21 +498,22 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 namespace fc {
 
 int attention_ws_launch(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const CUtensorMap& tq,
-                        const CUtensorMap& tk, const CUtensorMap& tv, void* O) {
+                        const CUtensorMap& tk, const CUtensorMap& tv, void* O, uint32_t* counter) {
   int max_items = 0;
   for (int c = 0; c < g.W; ++c) max_items += (g.q_row_off[c + 1] - g.q_row_off[c] + 2 * kBM - 1) / (2 * kBM);
   const int64_t items = (int64_t)max_items * g.H_q;
   if (items == 0) return FC_OK;
+  FC_CUDA_CHECK(cudaMemsetAsync(counter, 0, sizeof(uint32_t), st));
   const int grid = (int)std::min<int64_t>(items, (int64_t)ctx->sm_count);
   // at least half of the shared memory, so that a second CTA (and its 512 columns) never joins the SM
   const size_t need = (2 + 2 * kStages) * (size_t)kBM * g.d * 2 + sizeof(WsSmem) + 1024;
   const size_t smem = std::max<size_t>(need, 120 * 1024);
   if (g.d == 128) {
     FC_CUDA_CHECK(cudaFuncSetAttribute(attention_ws_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attention_ws_kernel<128><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O);
+    attention_ws_kernel<128><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O, counter);
   } else {
     FC_CUDA_CHECK(cudaFuncSetAttribute(attention_ws_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attention_ws_kernel<64><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O);
+    attention_ws_kernel<64><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O, counter);
   }
   FC_LAUNCH_CHECK("attention_ws_kernel");
   return FC_OK;

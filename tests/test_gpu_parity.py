@@ -195,13 +195,28 @@ def test_attention_token_index_map(ctx):
     _attention_case(ctx, wb, [1], token_map=True, atol=1e-2, rel_l2=1e-2)
 
 
-def test_attention_bf16_tensor_core_small(ctx):
+@pytest.mark.parametrize("impl", [2, 3])  # warp-specialised and single-stage tcgen05 kernels
+@pytest.mark.parametrize("d", [128, 64])
+def test_attention_bf16_tensor_core_small(ctx, impl, d):
     # several 128-row tiles with ragged tails in both rows and keys, a clean region and a window
-    w = wl.Workload("t", "bf16", H=2, d=128, W=3, n_c=328, B=200, L_k=528, seed=15, sigma=0.5)
-    _attention_case(ctx, w, [0, 1, 2], atol=1e-2, rel_l2=1e-2)
-    _attention_case(ctx, w, [2], atol=1e-2, rel_l2=1e-2)
-    w2 = wl.Workload("t2", "bf16", H=3, d=128, W=2, n_c=1000, B=0, L_k=1000, seed=16, sigma=0.5)
-    _attention_case(ctx, w2, [0, 1], atol=1e-2, rel_l2=1e-2)
+    w = wl.Workload("t", "bf16", H=2, d=d, W=3, n_c=328, B=200, L_k=528, seed=15, sigma=0.5)
+    _attention_case(ctx, w, [0, 1, 2], impl=impl, atol=1e-2, rel_l2=1e-2)
+    _attention_case(ctx, w, [2], impl=impl, atol=1e-2, rel_l2=1e-2)
+    w2 = wl.Workload("t2", "bf16", H=3, d=d, W=2, n_c=1000, B=0, L_k=1000, seed=16, sigma=0.5)
+    _attention_case(ctx, w2, [0, 1], impl=impl, atol=1e-2, rel_l2=1e-2)
+
+
+def test_attention_bf16_many_items_per_cta(ctx):
+    # more work items than SMs, of very different lengths: exercises the device-side item queue
+    w = wl.Workload("q", "bf16", H=40, d=128, W=6, n_c=520, B=300, L_k=820, seed=18, sigma=0.5)
+    _attention_case(ctx, w, [0, 1, 3, 5], impl=2, sample=wl.sample_rows(w, 40, 1), atol=1e-2, rel_l2=1e-2)
+
+
+@pytest.mark.parametrize("name,active", [("single_step_bf16", [0, 1, 2, 3]), ("cached_step_bf16", [2, 5, 7])])
+def test_attention_full_size_sampled_rows(ctx, name, active):
+    # the launch configuration the benchmark times, checked on sampled query rows over the full key range
+    w = wl.CONFIGS[name]
+    _attention_case(ctx, w, active, sample=wl.sample_rows(w, 48, 2), atol=1e-2, rel_l2=1e-2)
 
 
 def test_attention_bf16_matches_cuda_core_kernel(ctx):

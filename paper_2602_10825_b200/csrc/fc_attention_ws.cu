@@ -9,8 +9,8 @@
 //   warp  8    scheduler + TMA       takes the next item off the counter, publishes it to the
 //                                    other warps through a 2-slot ring, then loads the Q pair and
 //                                    streams K and V tiles into 2-stage rings
-//   warp  9    MMA issuer            S_A(j), PV_B(j-1), S_B(j), PV_A(j), ... so the tensor pipe
-//                                    always has the other tile's work while one tile is in softmax
+//   warps 9,10 MMA issuers           one thread per query tile: S_x(j), PV_x(j), S_x(j+1), ...; the tensor
+//                                    pipe runs the other tile's instructions while one tile is in softmax
 // Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512); P (bf16) overwrites the
 // low half of its S.  tcgen05.mma executes in issue order, so S_X(j+1) cannot overtake PV_X(j),
 // which still reads P_X(j), and "S_X(j) is complete" implies "PV_X(j-1) is complete", which is
@@ -32,8 +32,8 @@ namespace {
 using namespace fc::sm100;
 
 constexpr int kBM = 128, kBN = 128;
-constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {TMA warp, MMA warp, 2 spare warps}
-constexpr int kStages = 2;
+constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {copy warp, two MMA warps, a spare warp}
+constexpr int kStages = 2;  // the MMA issuer computes stage and phase with masks: keep at 2
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 // of every 32 columns, this many (the last ones) take the polynomial exponential
@@ -41,6 +41,30 @@ constexpr float kRescaleThreshold = 8.f;  // log2 units
 #define FC_ATTN_EMU_COLS 8
 #endif
 constexpr int kEmuCols = FC_ATTN_EMU_COLS;
+// Registers per thread after the split: softmax warpgroups / the warpgroup of the copy and MMA warps.
+// The CTA owns 384 x 168 registers from launch (168 = what the launch bounds allow); setmaxnreg only moves
+// registers inside that pool, and an increase that the pool cannot cover would wait forever.
+#ifndef FC_ATTN_REGS_HI
+#define FC_ATTN_REGS_HI 216
+#define FC_ATTN_REGS_LO 72
+#endif
+static_assert(256 * FC_ATTN_REGS_HI + 128 * FC_ATTN_REGS_LO <= 384 * 168, "register split exceeds the CTA's pool");
+static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg takes multiples of 8");
+// how whole warps (softmax, copy) wait on a barrier: 0 every lane polls, 1 lane 0 polls, 2 lane 0 with a short sleep
+#ifndef FC_ATTN_WARP_WAIT
+#define FC_ATTN_WARP_WAIT 0
+#endif
+#ifndef FC_ATTN_STAGGER
+#define FC_ATTN_STAGGER 1
+#endif
+constexpr bool kStagger = FC_ATTN_STAGGER != 0;
+// the pacing flag of a tile is raised after this 32-column chunk of its exponentials (0..3)
+#ifndef FC_ATTN_PACE_CHUNK
+#define FC_ATTN_PACE_CHUNK 0
+#endif
+constexpr int kPaceChunk = FC_ATTN_PACE_CHUNK;
+#define FC_STR2(x) #x
+#define FC_STR(x) FC_STR2(x)
 
 struct WsSmem {
   uint64_t q_full, q_empty;
@@ -48,6 +72,7 @@ struct WsSmem {
   uint64_t s_full[2], p_ready[2], o_done[2];
   uint64_t it_full[2], it_empty[2];
   int32_t it_slot[2];
+  uint32_t half_done[2];  // per query tile: key tiles whose softmax its first warp has half finished (pacing hint)
   uint32_t tmem_base;
   uint32_t abort;
   int32_t n_act, total_items;
@@ -114,7 +139,8 @@ __device__ __forceinline__ void ex2_poly2(float x0, float x1, float& y0, float& 
 
 // P = 2^(S * scale - m) for one row of a 128-column tile, written back over S as bf16; returns the row sum.
 template <bool kAllEx2>
-__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s) {
+__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s,
+                                          volatile uint32_t* half_flag, uint32_t half_value) {
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t sum2[2] = {0ull, 0ull};
   constexpr int kEmuPairs = kAllEx2 ? 0 : kEmuCols / 2;
@@ -137,11 +163,22 @@ __device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale
       pk[i] = cvt_bf16x2(p0, p1);
     }
     tmem_st16(t_s + q2 * 16, pk);
+    if (q2 == kPaceChunk && half_flag) *half_flag = half_value;  // this far through the tile
   }
   float a, b, c, d;
   unpack2(sum2[0], a, b);
   unpack2(sum2[1], c, d);
   return (a + b) + (c + d);
+}
+
+__device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort) {
+#if FC_ATTN_WARP_WAIT == 0
+  mbar_wait_bounded(bar, parity, abort);
+#elif FC_ATTN_WARP_WAIT == 1
+  mbar_wait_warp(bar, parity, abort, 0);
+#else
+  mbar_wait_warp(bar, parity, abort, 32);
+#endif
 }
 
 template <int D>
@@ -163,23 +200,24 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
 
   if (tid == 0) {
     mbar_init(smem_u32(&sh->q_full), 1);
-    mbar_init(smem_u32(&sh->q_empty), 1);
+    mbar_init(smem_u32(&sh->q_empty), 2);  // both MMA threads
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->k_full[s]), 1);
-      mbar_init(smem_u32(&sh->k_empty[s]), 1);
+      mbar_init(smem_u32(&sh->k_empty[s]), 2);  // both MMA threads
       mbar_init(smem_u32(&sh->v_full[s]), 1);
-      mbar_init(smem_u32(&sh->v_empty[s]), 1);
+      mbar_init(smem_u32(&sh->v_empty[s]), 2);
     }
     for (int x = 0; x < 2; ++x) {
       mbar_init(smem_u32(&sh->s_full[x]), 1);
       mbar_init(smem_u32(&sh->p_ready[x]), 4);  // one arrival per softmax warp
       mbar_init(smem_u32(&sh->o_done[x]), 1);
       mbar_init(smem_u32(&sh->it_full[x]), 1);
-      mbar_init(smem_u32(&sh->it_empty[x]), 9);  // the MMA warp and the eight softmax warps
+      mbar_init(smem_u32(&sh->it_empty[x]), 10);  // the two MMA threads and the eight softmax warps
       sh->it_slot[x] = -1;
     }
     mbar_fence_init();
     sh->abort = 0;
+    sh->half_done[0] = sh->half_done[1] = 0;
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
@@ -235,7 +273,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   // consumer side of the item ring; -1 once the list is exhausted or the CTA has given up
   auto next_item = [&](uint32_t n) {
     const int slot = n & 1;
-    mbar_wait_bounded(smem_u32(&sh->it_full[slot]), (n >> 1) & 1, abort);
+    warp_wait(smem_u32(&sh->it_full[slot]), (n >> 1) & 1, abort);
     int item = sh->it_slot[slot];
     __syncwarp();
     if (lane == 0) mbar_arrive(smem_u32(&sh->it_empty[slot]));
@@ -254,9 +292,9 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   };
 
   // Registers move from the third warpgroup, which only issues copies and MMAs, to the softmax
-  // warpgroups, which hold a 128-column row of S per thread: 256 x 224 + 128 x 56 <= 64 Ki.
+  // warpgroups, which hold a 128-column row of S per thread.
   if (warp >= 8) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 " FC_STR(FC_ATTN_REGS_LO) ";");
   if (warp == 8) {
     // ------------------------------------------------------------------ scheduler + TMA producer
     uint32_t kv = 0, it_n = 0;
@@ -266,7 +304,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       int item = __shfl_sync(0xffffffffu, next, 0);
       if (item >= total_items) item = -1;
       const int slot = it_n & 1;
-      mbar_wait_bounded(smem_u32(&sh->it_empty[slot]), ((it_n >> 1) & 1) ^ 1, abort);
+      warp_wait(smem_u32(&sh->it_empty[slot]), ((it_n >> 1) & 1) ^ 1, abort);
       if (lane == 0) {
         sh->it_slot[slot] = item < 0 ? total_items : item;
         mbar_arrive(smem_u32(&sh->it_full[slot]));
@@ -274,7 +312,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       if (item < 0 || *abort) break;
       if (lane == 0) next = (int)atomicAdd(counter, 1u);  // in flight while this item's tiles are loaded
       const Item it = decode(item);
-      mbar_wait_bounded(smem_u32(&sh->q_empty), (it_n & 1) ^ 1, abort);
+      warp_wait(smem_u32(&sh->q_empty), (it_n & 1) ^ 1, abort);
       if (lane == 0) {
         mbar_expect_tx(smem_u32(&sh->q_full), 2 * kTileBytes);
         for (int t = 0; t < 2; ++t)
@@ -287,14 +325,14 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         if (seg_vis <= 0) break;
         for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv) {
           const int st = kv % kStages, ph = (kv / kStages) & 1, prow = g.seg_phys[s] + j0;
-          mbar_wait_bounded(smem_u32(&sh->k_empty[st]), ph ^ 1, abort);
+          warp_wait(smem_u32(&sh->k_empty[st]), ph ^ 1, abort);
           if (lane == 0) {
             mbar_expect_tx(smem_u32(&sh->k_full[st]), kTileBytes);
             for (int x = 0; x < kAtoms; ++x)
               tma_load_3d(k_s + st * kTileBytes + x * kAtomBytes, &tmap_k, smem_u32(&sh->k_full[st]), x * 64, prow,
                           it.hk);
           }
-          mbar_wait_bounded(smem_u32(&sh->v_empty[st]), ph ^ 1, abort);
+          warp_wait(smem_u32(&sh->v_empty[st]), ph ^ 1, abort);
           if (lane == 0) {
             mbar_expect_tx(smem_u32(&sh->v_full[st]), kTileBytes);
             for (int x = 0; x < kAtoms; ++x)
@@ -306,85 +344,83 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
       ++it_n;
     }
-  } else if (warp == 9) {
-    // ------------------------------------------------------------------ MMA issuer
+  } else if (warp == 9 || warp == 10) {
+    // ------------------------------------------------------------------ MMA issuers (one thread per query tile)
+    // Lane 0 of warp 9 issues S_A and PV_A, lane 0 of warp 10 issues S_B and PV_B.  The tensor pipe takes
+    // instructions in arrival order; the order that matters, S_x(j+1) after PV_x(j), is program order of one
+    // thread.  While one thread sits in a wait or a commit the other keeps the pipe fed, and neither is held up
+    // by the other tile's softmax.
+    if (lane == 0) {
+    const int x = warp - 9;
     constexpr uint32_t kIdescQK = idesc_bf16_f32(kBM, kBN, false, false);
     constexpr uint32_t kIdescPV = idesc_bf16_f32(kBM, D, false, true);
-    auto issue_s = [&](int x, int st) {  // S_x = Q_x K^T
+    // descriptors are built once; a k-step only moves the 14-bit address field (units of 16 bytes)
+    const uint64_t dq = smem_desc_sw128(q_s + x * kTileBytes, 16, 1024), dk = smem_desc_sw128(k_s, 16, 1024),
+                   dv = smem_desc_sw128(v_s, kAtomBytes, 1024);
+    const uint32_t t_s = tmem + x * 128, t_o = tmem + 256 + x * 128;
+    auto issue_s = [&](uint32_t st) {  // S_x = Q_x K^T
+      const uint64_t b0 = dk + (uint64_t)(st * (kTileBytes >> 4));
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
-        const uint32_t off = (kk / 4) * kAtomBytes + (kk % 4) * 32;
-        umma_ss(tmem + x * 128, smem_desc_sw128(q_s + x * kTileBytes + off, 16, 1024),
-                smem_desc_sw128(k_s + st * kTileBytes + off, 16, 1024), kIdescQK, kk > 0);
+        const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
+        umma_ss(t_s, dq + off, b0 + off, kIdescQK, kk > 0);
       }
     };
-    auto issue_pv = [&](int x, int st, bool accumulate) {  // O_x (+)= P_x V
+    auto issue_pv = [&](uint32_t st, bool accumulate) {  // O_x (+)= P_x V
+      const uint64_t b0 = dv + (uint64_t)(st * (kTileBytes >> 4));
 #pragma unroll
       for (int kk = 0; kk < kBN / 16; ++kk)
-        umma_ts(tmem + 256 + x * 128, tmem + x * 128 + kk * 8,
-                smem_desc_sw128(v_s + st * kTileBytes + kk * 2048, kAtomBytes, 1024), kIdescPV, accumulate || kk > 0);
+        umma_ts(t_o, t_s + kk * 8, b0 + (uint64_t)(kk * (2048 >> 4)), kIdescPV, accumulate || kk > 0);
+    };
+    // barrier addresses as plain registers: the issue loop should be little more than the MMAs themselves
+    const uint32_t b_kfull = smem_u32(&sh->k_full[0]), b_kempty = smem_u32(&sh->k_empty[0]);
+    const uint32_t b_vfull = smem_u32(&sh->v_full[0]), b_vempty = smem_u32(&sh->v_empty[0]);
+    const uint32_t b_sfull = smem_u32(&sh->s_full[x]), b_pready = smem_u32(&sh->p_ready[x]);
+    // Pacing.  Left alone, the two tiles fall into step: both softmaxes run together, sharing the special-
+    // function unit, and then both tiles' MMAs queue up behind each other.  So each S is issued only once the
+    // other tile's softmax is half way through its current key tile: S_B(j) after half of softmax A(j), S_A(j+1)
+    // after half of softmax B(j).  That keeps the two softmaxes about half a period apart, and one tile's MMAs
+    // run under the other tile's softmax.  It is only a delay: no data depends on it, and it gives up after 20 us.
+    auto pace = [&](uint32_t want) {
+      if (!kStagger) return;
+      volatile uint32_t* other = &sh->half_done[x ^ 1];
+      if ((int32_t)(*other - want) >= 0) return;
+      const uint64_t t0 = global_timer_ns();
+      while ((int32_t)(*other - want) < 0 && global_timer_ns() - t0 < 20000ull) {
+      }
     };
     uint32_t kv = 0;
     for (uint32_t it_n = 0;; ++it_n) {
-      const int item = next_item(it_n);
-      if (item < 0) break;
+      const int slot = it_n & 1;
+      mbar_wait_bounded(smem_u32(&sh->it_full[slot]), (it_n >> 1) & 1, abort);
+      const int item = sh->it_slot[slot];
+      mbar_arrive(smem_u32(&sh->it_empty[slot]));
+      if (*abort || item >= total_items) break;
       const Item it = decode(item);
       const int n_tiles = count_tiles(it);
       mbar_wait_bounded(smem_u32(&sh->q_full), it_n & 1, abort);
       tc_fence_after();
-      if (n_tiles == 0 && lane == 0) umma_commit(smem_u32(&sh->q_empty));
-      int j = 0;  // tile index inside the item
-      for (int s = 0; s < g.n_seg; ++s) {
-        const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
-        if (seg_vis <= 0) break;
-        for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv, ++j) {
-          const int st = kv % kStages, ph = (kv / kStages) & 1;
-          mbar_wait_bounded(smem_u32(&sh->k_full[st]), ph, abort);
-          tc_fence_after();
-          if (lane == 0) {
-            issue_s(0, st);
-            umma_commit(smem_u32(&sh->s_full[0]));
-          }
-          if (j > 0) {  // PV_B of the previous tile
-            const uint32_t pkv = kv - 1;
-            mbar_wait_bounded(smem_u32(&sh->p_ready[1]), pkv & 1, abort);
-            tc_fence_after();
-            if (lane == 0) {
-              issue_pv(1, pkv % kStages, j > 1);
-              umma_commit(smem_u32(&sh->v_empty[pkv % kStages]));
-            }
-          }
-          if (lane == 0) {
-            issue_s(1, st);
-            umma_commit(smem_u32(&sh->s_full[1]));
-            umma_commit(smem_u32(&sh->k_empty[st]));
-            if (j == n_tiles - 1) umma_commit(smem_u32(&sh->q_empty));  // last read of the Q pair
-          }
-          mbar_wait_bounded(smem_u32(&sh->p_ready[0]), kv & 1, abort);
-          mbar_wait_bounded(smem_u32(&sh->v_full[st]), ph, abort);
-          tc_fence_after();
-          if (lane == 0) issue_pv(0, st, j > 0);
-          __syncwarp();
-        }
-      }
-      if (j > 0) {
-        const uint32_t pkv = kv - 1;
-        mbar_wait_bounded(smem_u32(&sh->p_ready[1]), pkv & 1, abort);
+      for (int j = 0; j < n_tiles; ++j, ++kv) {
+        const uint32_t st = kv & 1, ph = (kv >> 1) & 1;  // kStages == 2
+        mbar_wait_bounded(b_kfull + 8 * st, ph, abort);
+        pace(kv + x);
         tc_fence_after();
-        if (lane == 0) {
-          issue_pv(1, pkv % kStages, j > 1);
-          umma_commit(smem_u32(&sh->v_empty[pkv % kStages]));
-        }
+        issue_s(st);
+        umma_commit(b_sfull);
+        umma_commit(b_kempty + 8 * st);
+        mbar_wait_bounded(b_vfull + 8 * st, ph, abort);
+        mbar_wait_bounded(b_pready, kv & 1, abort);
+        tc_fence_after();
+        issue_pv(st, j > 0);
+        umma_commit(b_vempty + 8 * st);
       }
-      if (lane == 0) {
-        umma_commit(smem_u32(&sh->o_done[0]));
-        umma_commit(smem_u32(&sh->o_done[1]));
-      }
-      __syncwarp();
+      umma_commit(smem_u32(&sh->q_empty));  // every read of this thread's Q tile has been issued
+      umma_commit(smem_u32(&sh->o_done[x]));
+    }
     }
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 " FC_STR(FC_ATTN_REGS_HI) ";");
     // ------------------------------------------------------------------ softmax + epilogue, tile x
     const int x = warp >> 2;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -392,6 +428,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const uint32_t t_o = tmem + lane_base + 256 + x * 128;
     const int r_in = (warp & 3) * 32 + lane;  // row inside the tile
     const float scale_log2 = g.scale * 1.4426950408889634f;
+    volatile uint32_t* half_flag = (kStagger && (warp & 3) == 0 && lane == 0) ? &sh->half_done[x] : nullptr;
     uint32_t kv = 0;
     for (uint32_t it_n = 0;; ++it_n) {
       const int item = next_item(it_n);
@@ -404,7 +441,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         if (seg_vis <= 0) break;
         for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv, ++j) {
           const int cols_valid = min(kBN, seg_vis - j0);
-          mbar_wait_bounded(smem_u32(&sh->s_full[x]), kv & 1, abort);
+          warp_wait(smem_u32(&sh->s_full[x]), kv & 1, abort);
           tc_fence_after();
           uint32_t sv[kBN];
           tmem_ld128_wait(t_s, sv);
@@ -439,8 +476,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             }
           }
           // a ragged tile takes ex2 everywhere so that its masked columns give exactly 0
-          const float row_sum = cols_valid < kBN ? exp_tile<true>(sv, scale_log2, m, t_s)
-                                                 : exp_tile<false>(sv, scale_log2, m, t_s);
+          const float row_sum = cols_valid < kBN ? exp_tile<true>(sv, scale_log2, m, t_s, half_flag, kv + 1)
+                                                 : exp_tile<false>(sv, scale_log2, m, t_s, half_flag, kv + 1);
           l = l * alpha + row_sum;
           tmem_wait_st();
           tc_fence_before();
@@ -449,7 +486,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
       }
       // epilogue
-      mbar_wait_bounded(smem_u32(&sh->o_done[x]), it_n & 1, abort);
+      warp_wait(smem_u32(&sh->o_done[x]), it_n & 1, abort);
       tc_fence_after();
       const int row = it.row0 + x * kBM + r_in;
       const bool row_ok = row < g.q_row_off[it.c + 1];

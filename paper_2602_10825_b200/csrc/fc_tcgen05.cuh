@@ -40,19 +40,48 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Gives up after `limit` failed polls or as soon as another thread of the CTA has
-// given up (*abort != 0); the caller then runs on without waiting, so control flow stays uniform
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Bounded wait.  Gives up once `limit_ns` of wall time have passed (checked every 32 failed polls; one poll
+// may itself suspend the thread for a short, hardware-defined time) or as soon as another thread of the
+// CTA has given up (*abort != 0); the caller then runs on without waiting, so control flow stays uniform
 // and the kernel reaches its normal teardown.  Returns false if it gave up.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t* abort,
-                                                  uint32_t limit = (1u << 22)) {
+                                                  uint64_t limit_ns = 2000000000ull) {
   if (mbar_try_wait(bar, parity)) return true;
-  for (uint32_t n = 0; n < limit; ++n) {
+  const uint64_t t0 = global_timer_ns();
+  for (uint32_t n = 1;; ++n) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort) return false;
-    if (n > 64) __nanosleep(64);
+    if ((n & 31u) == 0 && global_timer_ns() - t0 > limit_ns) break;
   }
   *abort = 1;
   return false;
+}
+
+// The same wait for a whole warp: lane 0 polls and the other lanes park at the warp barrier, so a waiting
+// warp costs one thread's worth of polling.  `backoff_ns` > 0 sleeps between polls.
+__device__ __forceinline__ void mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort,
+                                               uint32_t backoff_ns = 0) {
+  if ((threadIdx.x & 31) == 0) {
+    if (!mbar_try_wait(bar, parity)) {
+      const uint64_t t0 = global_timer_ns();
+      for (uint32_t n = 1;; ++n) {
+        if (backoff_ns) __nanosleep(backoff_ns);
+        if (mbar_try_wait(bar, parity)) break;
+        if (*abort) break;
+        if ((n & 31u) == 0 && global_timer_ns() - t0 > 2000000000ull) {
+          *abort = 1;
+          break;
+        }
+      }
+    }
+  }
+  __syncwarp();
 }
 
 // ---- TMA ------------------------------------------------------------------------------------

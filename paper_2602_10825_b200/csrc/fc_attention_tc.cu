@@ -258,6 +258,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   if (warp == 0) tmem_dealloc(tmem, kTmemCols);
 }
 
+}  // namespace
+
+namespace fc {
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -280,9 +284,6 @@ int make_tmap(fc_ctx* ctx, CUtensorMap* map, const void* base, int d, int64_t ro
   return FC_OK;
 }
 
-}  // namespace
-
-namespace fc {
 
 size_t attention_tc_workspace_bytes() { return 256; }
 

@@ -1,6 +1,9 @@
 // fc_kv_score: importance (Eq. 9), max-pool (Eq. 10), redundancy (Eq. 11, through the mean-key
 // identity of the paper's efficiency appendix) and the mixed score (Eq. 12).
 //
+// Two pipelines, both deterministic (no floating-point atomics).  bf16 inputs with one query head per key head
+// and at most 64 observation queries take the tensor-core kernels of fc_score_tc.cu followed by the finalize
+// kernel below; everything else (fp32, grouped query heads, more queries) takes the
 // CUDA-core pipeline, deterministic (no floating-point atomics), five launches per call:
 //   pass1     one thread per key: raw logits of all observation queries against its key,
 //             written to the workspace; normalised key summed per 128-key tile (mean key)
@@ -13,6 +16,7 @@
 #include <cmath>
 
 #include "fc_common.cuh"
+#include "fc_score.cuh"
 
 namespace {
 
@@ -244,6 +248,9 @@ score_finalize_kernel(ScoreGeom g, const float* __restrict__ imp_in, const float
 struct ScoreWs {
   float *S, *mk_partial, *lse, *mean_key, *a, *imp_tmp;
   float2* a_partial;
+  float2* tc_ml;      // tensor-core path: per-slice (max, sum) of every query
+  float* tc_colsum;   // per-slice sums of normalised keys
+  float* tc_lse2;
   size_t total;
 };
 
@@ -262,6 +269,9 @@ ScoreWs carve(const ScoreGeom& g, void* ws) {
   w.a = (float*)take((size_t)g.H_kv * g.L_k * 4);
   w.imp_tmp = (float*)take((size_t)g.H_kv * g.L_k * 4);
   w.a_partial = (float2*)take((size_t)g.H_kv * g.n_tiles * 8);
+  w.tc_ml = (float2*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * fc::kScoreTcMaxQueries * 8);
+  w.tc_colsum = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * g.d * 4);
+  w.tc_lse2 = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxQueries * 4);
   w.total = off;
   return w;
 }
@@ -319,7 +329,6 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
                            const void* K_cand, int dtype, float* imp_accum, int accum_phase, int n_steps,
                            float* imp, float* red, float* score, uint32_t* status, void* ws,
                            size_t ws_bytes) {
-  (void)status;
   if (!ctx || !Q_obs || !K_cand) return FC_ERR_INVALID_ARG;
   ScoreGeom g;
   int rc = make_geom(desc, g);
@@ -337,6 +346,23 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
   if (!ws || ws_bytes < w.total) return FC_ERR_WORKSPACE;
   if (!fc::aligned16(ws)) return FC_ERR_MISALIGNED;
   cudaStream_t st = (cudaStream_t)stream;
+  if (desc->impl < 0 || desc->impl > 2) return FC_ERR_INVALID_ARG;
+  const bool tc_ok = dtype == FC_BF16 && g.group == 1 && g.L_q <= fc::kScoreTcMaxQueries;
+  if (desc->impl == 2 && !tc_ok) return FC_ERR_UNSUPPORTED;
+  if (tc_ok && desc->impl != 1) {
+    fc::ScoreTcArgs a;
+    a.H = g.H_kv; a.L_q = g.L_q; a.L_k = g.L_k; a.n_tiles = g.n_tiles; a.tiles_per_slice = 0; a.n_slices = 0;
+    a.scale_log2 = g.scale * 1.4426950408889634f;
+    a.accum_phase = accum_phase; a.n_steps = n_steps;
+    a.ml_part = w.tc_ml; a.colsum_part = w.tc_colsum; a.lse2 = w.tc_lse2; a.mean_key = w.mean_key;
+    a.imp_accum = imp_accum; a.imp_out = imp ? imp : w.imp_tmp; a.a_out = w.a; a.a_partial = w.a_partial;
+    a.status = status;
+    rc = fc::score_tc_run(ctx, st, a, g.d, g.q_hs, g.q_rs, g.k_hs, g.k_rs, Q_obs, K_cand);
+    if (rc != FC_OK || accum_phase == 1) return rc;
+    score_finalize_kernel<<<dim3(g.n_tiles, g.H_kv), kTile, 0, st>>>(g, a.imp_out, w.a, w.a_partial, red, score);
+    FC_LAUNCH_CHECK("score_finalize_kernel");
+    return FC_OK;
+  }
   if (dtype == FC_BF16) {
     if (g.d == 128) return run<__nv_bfloat16, 128>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
     return run<__nv_bfloat16, 64>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);

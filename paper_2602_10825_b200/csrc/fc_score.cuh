@@ -1,0 +1,32 @@
+// Interface between fc_kv_score's front end (fc_score.cu) and its tensor-core kernels (fc_score_tc.cu).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "fc_common.cuh"
+
+namespace fc {
+
+constexpr int kScoreTcMaxQueries = 64;  // observation queries the tensor-core path takes (zero-padded to this)
+constexpr int kScoreTcMaxSlices = 64;   // slices of key tiles per head
+
+struct ScoreTcArgs {
+  int H, L_q, L_k, n_tiles, tiles_per_slice, n_slices;  // n_tiles = ceil(L_k / 128); slices are set by score_tc_run
+  float scale_log2;                                     // softmax scale times log2(e)
+  int accum_phase, n_steps;
+  float2* ml_part;     // [H, n_slices, 64] running (max, sum) of pass 1, log2 domain
+  float* colsum_part;  // [H, n_slices, d] sums of normalised keys
+  float* lse2;         // [H, 64]
+  float* mean_key;     // [H, d]
+  float* imp_accum;    // caller's accumulator or NULL
+  float* imp_out;      // [H, L_k]
+  float* a_out;        // [H, L_k] redundancy logits
+  float2* a_partial;   // [H, n_tiles] softmax statistics of a per 128-key tile
+  uint32_t* status;
+};
+
+// pass 1, merge, pass 2; the caller runs the finalize kernel afterwards (unless accum_phase == 1)
+int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs args, int d, int64_t q_hs, int64_t q_rs, int64_t k_hs,
+                 int64_t k_rs, const void* Q, const void* K);
+
+}  // namespace fc

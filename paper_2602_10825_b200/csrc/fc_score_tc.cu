@@ -1,0 +1,400 @@
+// fc_kv_score on tcgen05 tensor cores (bf16 keys and queries, one query head per key head, at most 64
+// observation queries).
+//
+// The importance of a key is a column sum of a row-normalised matrix (Eq. 9), so the logits are needed
+// twice: once to get every query's log-sum-exp over all candidates, once to add up exp(logit - lse) per key.
+// Both passes recompute the logits on the tensor cores instead of storing them (50 x L_k fp32 per head would be
+// five times the keys themselves), and each pass picks the orientation whose reduction stays inside a thread:
+//   pass 1  S[query, key] = Q K^T   one query row per thread: running (max, sum) over the keys of the slice;
+//                                   the same pass adds up the l2-normalised keys (the mean key of the
+//                                   paper's efficiency appendix)
+//   merge   per head: slices' (max, sum) -> log-sum-exp per query; slice sums -> mean normalised key
+//   pass 2  S[key, query] = K Q^T   one key row per thread: attention mass of the key; redundancy logit
+//                                   a_j = meankey . khat_j - |khat_j|^2 / L_k and its per-tile softmax statistics
+// The finalize step (softmax of a, max-pool, lambda-mix) is the one the CUDA-core path uses.
+//
+// A CTA owns one (head, slice of key tiles).  Warps 0-3 read the logits from tensor memory, warps 4-7 read the
+// key tile from shared memory (norms, column sums, dot with the mean key), warp 8 streams key tiles through a
+// 4-stage TMA ring and issues the MMAs into a 2-deep tensor-memory ring.  Keys are read from HBM once: the
+// second pass finds them in L2 for the cache sizes of the paper (a head is a few MB).
+// Sums are fixed-order: results are bit-reproducible from run to run.  Every mbarrier wait is bounded.
+#include <cmath>
+
+#include "fc_attention.cuh"
+#include "fc_score.cuh"
+#include "fc_tcgen05.cuh"
+#include "fc_tcgen05_ld.cuh"
+
+namespace {
+
+using namespace fc::sm100;
+
+constexpr int kKeys = 128;     // keys per tile
+constexpr int kRing = 4;       // key tiles in flight
+constexpr int kThreads = 288;  // warps 0-3 logits, warps 4-7 key vectors, warp 8 copies and MMAs
+constexpr int kNQ = fc::kScoreTcMaxQueries;  // queries of pass 2 (MMA N), zero-padded
+
+struct TcSmem {
+  uint64_t q_full, k_full[kRing], k_free[kRing], s_full[2], s_free[2];
+  uint32_t tmem_base, abort;
+  float inv_s[2][kKeys];   // 1 / |k| of the current tile's keys (double-buffered by tile parity)
+  float vec_s[128];        // pass 2: mean normalised key
+  float lse_s[kNQ];        // pass 2: log2-domain log-sum-exp per query
+  float red_m[2][4], red_l[2][4];
+  float colsum_s[16][128];  // pass 1: per row-group column sums at the end of the slice
+};
+
+// 16-byte chunk `c` of key row `r` inside a 128-byte-swizzled tile of 64-element column blocks
+template <int D>
+__device__ __forceinline__ uint4 lds_key_chunk(const uint8_t* tile, int r, int c) {
+  const int x = c >> 3, cc = c & 7;
+  return *reinterpret_cast<const uint4*>(tile + x * (kKeys * 128) + r * 128 + ((cc ^ (r & 7)) << 4));
+}
+
+__device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// PASS 1: ml_part [H, n_slices, kNQ] (max, sum) in the log2 domain; colsum_part [H, n_slices, D]
+// PASS 2: imp / a / a_partial as in the CUDA-core path
+template <int D, int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                const fc::ScoreTcArgs g) {
+  constexpr uint32_t kTileBytes = kKeys * D * 2;
+  constexpr int kAtoms = D / 64;
+  constexpr uint32_t kAtomBytes = kKeys * 128;
+  constexpr int kCols = PASS == 1 ? kKeys : kNQ;  // tensor-memory columns of one logit buffer
+  constexpr int kChunks = D / 8;                  // 16-byte chunks per key row
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* q_tile = smem;
+  uint8_t* k_tiles = smem + kTileBytes;
+  TcSmem* sh = (TcSmem*)(smem + (1 + kRing) * kTileBytes);
+  volatile uint32_t* abort = &sh->abort;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int hk = blockIdx.y, slice = blockIdx.x;
+  const int t0 = slice * g.tiles_per_slice, t1 = min(g.n_tiles, t0 + g.tiles_per_slice), n = t1 - t0;
+
+  if (tid == 0) {
+    mbar_init(smem_u32(&sh->q_full), 1);
+    for (int s = 0; s < kRing; ++s) {
+      mbar_init(smem_u32(&sh->k_full[s]), 1);
+      mbar_init(smem_u32(&sh->k_free[s]), 5);  // the MMA's commit and warps 4-7
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sh->s_full[b]), 1);
+      mbar_init(smem_u32(&sh->s_free[b]), 4);  // warps 0-3
+    }
+    mbar_fence_init();
+    sh->abort = 0;
+    tma_prefetch_desc(&tmap_q);
+    tma_prefetch_desc(&tmap_k);
+  }
+  if (PASS == 2) {
+    if (tid < D) sh->vec_s[tid] = g.mean_key[hk * D + tid];
+    if (tid < kNQ) sh->lse_s[tid] = g.lse2[hk * kNQ + tid];
+  }
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&sh->tmem_base), 2 * kCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh->tmem_base;
+
+  if (warp == 8) {
+    // ---------------------------------------------------------------- copies and MMAs (one thread)
+    if (lane == 0 && n > 0) {
+      auto load_k = [&](int i) {  // tile t0 + i into stage i % kRing
+        const int st = i % kRing;
+        const uint32_t bar = smem_u32(&sh->k_full[st]);
+        mbar_expect_tx(bar, kTileBytes);
+        for (int x = 0; x < kAtoms; ++x)
+          tma_load_3d(smem_u32(k_tiles + st * kTileBytes + x * kAtomBytes), &tmap_k, bar, x * 64, (t0 + i) * kKeys, hk);
+      };
+      mbar_expect_tx(smem_u32(&sh->q_full), kTileBytes);
+      for (int x = 0; x < kAtoms; ++x)
+        tma_load_3d(smem_u32(q_tile + x * kAtomBytes), &tmap_q, smem_u32(&sh->q_full), x * 64, 0, hk);
+      for (int i = 0; i < min(n, kRing - 1); ++i) load_k(i);
+      mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
+      const uint64_t dq = smem_desc_sw128(smem_u32(q_tile), 16, 1024);
+      constexpr uint32_t kIdesc = PASS == 1 ? idesc_bf16_f32(128, kKeys, false, false) : idesc_bf16_f32(kKeys, kNQ, false, false);
+      for (int i = 0; i < n; ++i) {
+        const int st = i % kRing, b = i & 1;
+        mbar_wait_bounded(smem_u32(&sh->k_full[st]), (i / kRing) & 1, abort);
+        mbar_wait_bounded(smem_u32(&sh->s_free[b]), ((i >> 1) & 1) ^ 1, abort);
+        tc_fence_after();
+        const uint64_t dk = smem_desc_sw128(smem_u32(k_tiles + st * kTileBytes), 16, 1024);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
+          if (PASS == 1) umma_ss(tmem + b * kCols, dq + off, dk + off, kIdesc, kk > 0);  // S[query, key]
+          else umma_ss(tmem + b * kCols, dk + off, dq + off, kIdesc, kk > 0);            // S[key, query]
+        }
+        umma_commit(smem_u32(&sh->s_full[b]));
+        umma_commit(smem_u32(&sh->k_free[st]));
+        if (i + kRing - 1 < n) {  // refill the stage tile i-1 has left
+          if (i >= 1) mbar_wait_bounded(smem_u32(&sh->k_free[(i - 1) % kRing]), ((i - 1) / kRing) & 1, abort);
+          load_k(i + kRing - 1);
+        }
+      }
+    }
+  } else if (warp < 4) {
+    // ---------------------------------------------------------------- logits out of tensor memory
+    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    if (PASS == 1) {
+      const int q = tid;  // query row
+      const bool row_ok = q < g.L_q;
+      const bool warp_ok = warp * 32 < g.L_q;
+      float m = -INFINITY, l = 0.f;
+      for (int i = 0; i < n; ++i) {
+        const int b = i & 1;
+        mbar_wait_bounded(smem_u32(&sh->s_full[b]), (i >> 1) & 1, abort);
+        tc_fence_after();
+        uint32_t sv[kKeys];
+        if (warp_ok) tmem_ld128_wait(t_lane + b * kCols, sv);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
+        if (!warp_ok) continue;
+        const int cols_valid = min(kKeys, g.L_k - (t0 + i) * kKeys);
+        if (cols_valid < kKeys) {
+#pragma unroll
+          for (int c = 0; c < kKeys; ++c)
+            if (c >= cols_valid) sv[c] = 0xff800000u;  // -inf
+        }
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int c = 0; c < kKeys; c += 8) {
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4)
+            mx[c4] = max3(mx[c4], __uint_as_float(sv[c + 2 * c4]), __uint_as_float(sv[c + 2 * c4 + 1]));
+        }
+        const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * g.scale_log2;  // scale > 0
+        if (tile_max > m) {
+          l *= ex2(m - tile_max);  // 0 on the first tile
+          m = tile_max;
+        }
+        const uint64_t sc2 = pack2(g.scale_log2, g.scale_log2), nm2 = pack2(-m, -m);
+        uint64_t sum2[2] = {0ull, 0ull};
+#pragma unroll
+        for (int c = 0; c < kKeys; c += 2) {
+          const uint64_t x = fma2(pack2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), sc2, nm2);
+          float x0, x1;
+          unpack2(x, x0, x1);
+          sum2[(c >> 1) & 1] = add2(sum2[(c >> 1) & 1], pack2(ex2(x0), ex2(x1)));
+        }
+        float a0, a1, a2, a3;
+        unpack2(sum2[0], a0, a1);
+        unpack2(sum2[1], a2, a3);
+        l += (a0 + a1) + (a2 + a3);
+      }
+      if (row_ok) g.ml_part[((int64_t)hk * g.n_slices + slice) * kNQ + q] = make_float2(m, l);
+    } else {
+      const float inv_nq = 1.f / (float)g.L_q;
+      for (int i = 0; i < n; ++i) {
+        const int b = i & 1;
+        mbar_wait_bounded(smem_u32(&sh->s_full[b]), (i >> 1) & 1, abort);
+        tc_fence_after();
+        uint32_t sv[kNQ];
+        tmem_ld64_wait(t_lane + b * kCols, sv);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
+        const int j = (t0 + i) * kKeys + tid;  // this thread's key
+        float mass = 0.f;
+#pragma unroll
+        for (int q = 0; q < kNQ; ++q)
+          if (q < g.L_q) mass += ex2(fmaf(__uint_as_float(sv[q]), g.scale_log2, -sh->lse_s[q]));
+        mass *= inv_nq;
+        if (j < g.L_k) {
+          const int64_t o = (int64_t)hk * g.L_k + j;
+          if (g.accum_phase == 1) {
+            g.imp_accum[o] += mass;
+          } else if (g.accum_phase == 2) {
+            const float t = g.imp_accum[o] + mass;
+            g.imp_accum[o] = t;
+            g.imp_out[o] = t / (float)g.n_steps;
+          } else {
+            g.imp_out[o] = mass;
+          }
+        }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- key vectors out of shared memory
+    const int u = tid - 128;  // 0..127
+    if (PASS == 1) {
+      // column sums of the normalised keys: this thread owns 16-byte chunk `c` of the rows r = rg (mod kGroups)
+      constexpr int kGroups = 128 / kChunks;  // 8 for d = 128, 16 for d = 64
+      const int c = u % kChunks, rg = u / kChunks;
+      float acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+      for (int i = 0; i < n; ++i) {
+        const int st = i % kRing;
+        mbar_wait_bounded(smem_u32(&sh->k_full[st]), (i / kRing) & 1, abort);
+        const uint8_t* tile = k_tiles + st * kTileBytes;
+        float n2 = 0.f;
+#pragma unroll
+        for (int cc = 0; cc < kChunks; ++cc) {
+          const uint4 w = lds_key_chunk<D>(tile, u, cc);
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float lo = fc::bf16_lo(ww[e]), hi = fc::bf16_hi(ww[e]);
+            n2 = fmaf(lo, lo, n2);
+            n2 = fmaf(hi, hi, n2);
+          }
+        }
+        // rows past the end of the cache are zero-filled: 0 * (1 / 1e-12) = 0, they add nothing
+        sh->inv_s[i & 1][u] = 1.f / fmaxf(sqrtf(n2), 1e-12f);
+        named_barrier_128();
+        for (int r = rg; r < kKeys; r += kGroups) {
+          const uint4 w = lds_key_chunk<D>(tile, r, c);
+          const float inv = sh->inv_s[i & 1][r];
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            acc[2 * e] = fmaf(fc::bf16_lo(ww[e]), inv, acc[2 * e]);
+            acc[2 * e + 1] = fmaf(fc::bf16_hi(ww[e]), inv, acc[2 * e + 1]);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh->k_free[st]));
+      }
+#pragma unroll
+      for (int e = 0; e < 8; ++e) sh->colsum_s[rg][c * 8 + e] = acc[e];
+      named_barrier_128();
+      if (u < D) {
+        float t = 0.f;
+        for (int r = 0; r < kGroups; ++r) t += sh->colsum_s[r][u];
+        g.colsum_part[((int64_t)hk * g.n_slices + slice) * D + u] = t;
+      }
+    } else {
+      for (int i = 0; i < n; ++i) {
+        const int st = i % kRing;
+        mbar_wait_bounded(smem_u32(&sh->k_full[st]), (i / kRing) & 1, abort);
+        const int tile_id = t0 + i, j = tile_id * kKeys + u;
+        const bool valid = j < g.L_k;
+        float a = -INFINITY;
+        if (g.accum_phase != 1) {
+          const uint8_t* tile = k_tiles + st * kTileBytes;
+          float n2 = 0.f, dot = 0.f;
+#pragma unroll
+          for (int cc = 0; cc < kChunks; ++cc) {
+            const uint4 w = lds_key_chunk<D>(tile, u, cc);
+            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+            const float4 m0 = *reinterpret_cast<const float4*>(&sh->vec_s[cc * 8]);
+            const float4 m1 = *reinterpret_cast<const float4*>(&sh->vec_s[cc * 8 + 4]);
+            const float mk[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float lo = fc::bf16_lo(ww[e]), hi = fc::bf16_hi(ww[e]);
+              n2 = fmaf(lo, lo, n2);
+              n2 = fmaf(hi, hi, n2);
+              dot = fmaf(mk[2 * e], lo, dot);
+              dot = fmaf(mk[2 * e + 1], hi, dot);
+            }
+          }
+          if (valid) {
+            const float inv = 1.f / fmaxf(sqrtf(n2), 1e-12f);
+            a = dot * inv - (n2 * inv * inv) / (float)g.L_k;
+            g.a_out[(int64_t)hk * g.L_k + j] = a;
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh->k_free[st]));
+        if (g.accum_phase == 1) continue;
+        // softmax statistics of a over the tile, fixed tree
+        float m = a, l = valid ? 1.f : 0.f;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float m2 = __shfl_down_sync(0xffffffffu, m, o), l2 = __shfl_down_sync(0xffffffffu, l, o);
+          const float mn = fmaxf(m, m2);
+          l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
+          m = mn;
+        }
+        if (lane == 0) {
+          sh->red_m[i & 1][warp - 4] = m;
+          sh->red_l[i & 1][warp - 4] = l;
+        }
+        named_barrier_128();
+        if (u == 0) {
+          m = sh->red_m[i & 1][0];
+          l = sh->red_l[i & 1][0];
+          for (int w = 1; w < 4; ++w) {
+            const float m2 = sh->red_m[i & 1][w], l2 = sh->red_l[i & 1][w];
+            const float mn = fmaxf(m, m2);
+            l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
+            m = mn;
+          }
+          g.a_partial[hk * g.n_tiles + tile_id] = make_float2(m, l);
+        }
+      }
+    }
+  }
+
+  if (*abort) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let copies and MMAs in flight land before teardown
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *abort && g.status) atomicOr(g.status, FC_DEV_TIMEOUT);
+  if (warp == 0) tmem_dealloc(tmem, 2 * kCols);
+}
+
+// per head: slices' (max, sum) -> log2-domain log-sum-exp per query; slices' column sums -> mean normalised key
+__global__ void score_tc_merge_kernel(const fc::ScoreTcArgs g, int d) {
+  const int hk = blockIdx.x, t = threadIdx.x;
+  if (t < kNQ) {
+    float lse = 0.f;
+    if (t < g.L_q) {
+      float m = -INFINITY, l = 0.f;
+      for (int s = 0; s < g.n_slices; ++s) {
+        const float2 p = g.ml_part[((int64_t)hk * g.n_slices + s) * kNQ + t];
+        const float mn = fmaxf(m, p.x);
+        l = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * exp2f(p.x - mn));
+        m = mn;
+      }
+      lse = m + log2f(l);
+    }
+    g.lse2[hk * kNQ + t] = lse;
+  }
+  if (t < d) {
+    float acc = 0.f;
+    for (int s = 0; s < g.n_slices; ++s) acc += g.colsum_part[((int64_t)hk * g.n_slices + s) * d + t];
+    g.mean_key[hk * d + t] = acc / (float)g.L_k;
+  }
+}
+
+}  // namespace
+
+namespace fc {
+
+int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs g, int d, int64_t q_hs, int64_t q_rs, int64_t k_hs,
+                 int64_t k_rs, const void* Q, const void* K) {
+  CUtensorMap tq, tk;
+  int rc;
+  if ((rc = make_tmap(ctx, &tq, Q, d, g.L_q, g.H, q_rs, g.H > 1 ? q_hs : q_rs * g.L_q)) != FC_OK) return rc;
+  if ((rc = make_tmap(ctx, &tk, K, d, g.L_k, g.H, k_rs, g.H > 1 ? k_hs : k_rs * g.L_k)) != FC_OK) return rc;
+  // slices: about two CTAs per SM over all heads, at most kScoreTcMaxSlices per head
+  const int want = std::max(1, (2 * ctx->sm_count + g.H - 1) / g.H);
+  g.n_slices = std::min(std::min(want, kScoreTcMaxSlices), g.n_tiles);
+  g.tiles_per_slice = (g.n_tiles + g.n_slices - 1) / g.n_slices;
+  g.n_slices = (g.n_tiles + g.tiles_per_slice - 1) / g.tiles_per_slice;  // no empty slice
+  const size_t smem = (size_t)(1 + kRing) * kKeys * d * 2 + sizeof(TcSmem) + 1024;
+  const dim3 grid(g.n_slices, g.H);
+  auto launch = [&](auto kernel) -> int {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<grid, kThreads, smem, st>>>(tq, tk, g);
+    FC_LAUNCH_CHECK("score_tc_kernel");
+    return FC_OK;
+  };
+  if ((rc = d == 128 ? launch(score_tc_kernel<128, 1>) : launch(score_tc_kernel<64, 1>)) != FC_OK) return rc;
+  score_tc_merge_kernel<<<g.H, 128, 0, st>>>(g, d);
+  FC_LAUNCH_CHECK("score_tc_merge_kernel");
+  return d == 128 ? launch(score_tc_kernel<128, 2>) : launch(score_tc_kernel<64, 2>);
+}
+
+}  // namespace fc

@@ -250,12 +250,34 @@ def test_score_tiny_f32_config(ctx):
     _score_case(ctx, Q_obs, K, w.lam, w.pool_k)
 
 
+@pytest.mark.parametrize("impl", [1, 2])  # CUDA-core and tensor-core pipelines
 @pytest.mark.parametrize("keys", ["normal", "clustered"])
-def test_score_bf16_ragged(ctx, keys):
+def test_score_bf16_ragged(ctx, keys, impl):
     w = wl.Workload("s", "bf16", H=3, d=128, W=1, n_c=100, B=1000, L_k=1331, seed=21, sigma=0.5, keys=keys)
     Q_obs, K, _ = wl.candidates(w)
-    _score_case(ctx, Q_obs, K, 0.07, 7)
-    _score_case(ctx, Q_obs, K, 0.5, 1)
+    _score_case(ctx, Q_obs, K, 0.07, 7, impl=impl)
+    _score_case(ctx, Q_obs, K, 0.5, 1, impl=impl)
+
+
+@pytest.mark.parametrize("d,L_q,L_k", [(64, 50, 777), (128, 64, 128), (128, 1, 5000), (128, 33, 9000)])
+def test_score_tensor_core_shapes(ctx, d, L_q, L_k):
+    # d = 64; exactly one tile; a single query; many tiles per slice with a ragged tail
+    Q = wl.normal((2, L_q, d), 51, 0.7, torch.bfloat16)
+    K = wl.normal((2, L_k, d), 52, 0.7, torch.bfloat16)
+    K[1, 5] = 0  # a zero key: its normalised form is 0
+    _score_case(ctx, Q, K, 0.07, 7, impl=2)
+
+
+def test_score_tensor_core_matches_cuda_core_full_size(ctx):
+    # config 3's compression event: both pipelines on every element
+    w = wl.CONFIGS["cached_step_bf16"]
+    Q_obs, K, _ = wl.candidates(w)
+    a = ctx.kv_score(dev(Q_obs), dev(K), lambda_=w.lam, pool_k=w.pool_k, impl=1)["score"]
+    b = ctx.kv_score(dev(Q_obs), dev(K), lambda_=w.lam, pool_k=w.pool_k, impl=2)["score"]
+    torch.cuda.synchronize()
+    assert (a - b).abs().max().item() <= 1e-4 * a.abs().max().item()
+    want = oracle.kv_score(wl.bits(Q_obs), wl.bits(K), lambda_=w.lam, pool_k=w.pool_k)["score"]
+    assert np.abs(b.double().cpu().numpy() - want).max() <= 1e-4 * np.abs(want).max()
 
 
 def test_score_gqa_and_d64(ctx):

@@ -2,7 +2,7 @@
 // identity of the paper's efficiency appendix) and the mixed score (Eq. 12).
 //
 // Two pipelines, both deterministic (no floating-point atomics).  bf16 inputs with one query head per key head
-// and at most 64 observation queries take the tensor-core kernels of fc_score_tc.cu followed by the finalize
+// and at most 62 observation queries take the tensor-core kernels of fc_score_tc.cu followed by the finalize
 // kernel below; everything else (fp32, grouped query heads, more queries) takes the
 // CUDA-core pipeline, deterministic (no floating-point atomics), five launches per call:
 //   pass1     one thread per key: raw logits of all observation queries against its key,
@@ -251,6 +251,7 @@ struct ScoreWs {
   float2* tc_ml;      // tensor-core path: per-slice (max, sum) of every query
   float* tc_colsum;   // per-slice sums of normalised keys
   float* tc_lse2;
+  float* tc_norm2;
   size_t total;
 };
 
@@ -272,6 +273,7 @@ ScoreWs carve(const ScoreGeom& g, void* ws) {
   w.tc_ml = (float2*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * fc::kScoreTcMaxQueries * 8);
   w.tc_colsum = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * g.d * 4);
   w.tc_lse2 = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxQueries * 4);
+  w.tc_norm2 = (float*)take((size_t)g.H_kv * g.L_k * 4);
   w.total = off;
   return w;
 }
@@ -347,14 +349,14 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
   if (!fc::aligned16(ws)) return FC_ERR_MISALIGNED;
   cudaStream_t st = (cudaStream_t)stream;
   if (desc->impl < 0 || desc->impl > 2) return FC_ERR_INVALID_ARG;
-  const bool tc_ok = dtype == FC_BF16 && g.group == 1 && g.L_q <= fc::kScoreTcMaxQueries;
+  const bool tc_ok = dtype == FC_BF16 && g.group == 1 && g.L_q <= fc::kScoreTcMaxQueries - 2;
   if (desc->impl == 2 && !tc_ok) return FC_ERR_UNSUPPORTED;
   if (tc_ok && desc->impl != 1) {
     fc::ScoreTcArgs a;
     a.H = g.H_kv; a.L_q = g.L_q; a.L_k = g.L_k; a.n_tiles = g.n_tiles; a.tiles_per_slice = 0; a.n_slices = 0;
     a.scale_log2 = g.scale * 1.4426950408889634f;
     a.accum_phase = accum_phase; a.n_steps = n_steps;
-    a.ml_part = w.tc_ml; a.colsum_part = w.tc_colsum; a.lse2 = w.tc_lse2; a.mean_key = w.mean_key;
+    a.ml_part = w.tc_ml; a.colsum_part = w.tc_colsum; a.lse2 = w.tc_lse2; a.mean_key = w.mean_key; a.norm2 = w.tc_norm2;
     a.imp_accum = imp_accum; a.imp_out = imp ? imp : w.imp_tmp; a.a_out = w.a; a.a_partial = w.a_partial;
     a.status = status;
     rc = fc::score_tc_run(ctx, st, a, g.d, g.q_hs, g.q_rs, g.k_hs, g.k_rs, Q_obs, K_cand);

@@ -7,7 +7,8 @@
 
 namespace fc {
 
-constexpr int kScoreTcMaxQueries = 64;  // observation queries the tensor-core path takes (zero-padded to this)
+constexpr int kScoreTcMaxQueries = 64;  // query rows of the tensor-core path: observation queries (at most 62, zero-
+                                        // padded) and two rows for the mean key
 constexpr int kScoreTcMaxSlices = 64;   // slices of key tiles per head
 
 struct ScoreTcArgs {
@@ -18,6 +19,7 @@ struct ScoreTcArgs {
   float* colsum_part;  // [H, n_slices, d] sums of normalised keys
   float* lse2;         // [H, 64]
   float* mean_key;     // [H, d]
+  float* norm2;        // [H, L_k] squared l2 norm of every key (pass 1 -> pass 2)
   float* imp_accum;    // caller's accumulator or NULL
   float* imp_out;      // [H, L_k]
   float* a_out;        // [H, L_k] redundancy logits

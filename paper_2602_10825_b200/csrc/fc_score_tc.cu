@@ -10,11 +10,15 @@
 //                                   paper's efficiency appendix)
 //   merge   per head: slices' (max, sum) -> log-sum-exp per query; slice sums -> mean normalised key
 //   pass 2  S[key, query] = K Q^T   one key row per thread: attention mass of the key; redundancy logit
-//                                   a_j = meankey . khat_j - |khat_j|^2 / L_k and its per-tile softmax statistics
+//                                   a_j = meankey . khat_j - |khat_j|^2 / L_k and its per-tile softmax statistics.
+//                                   The mean key rides along as two more query rows (its bf16 high and low
+//                                   parts: the keys are bf16, so the products are exact and the sum carries 16
+//                                   bits of the mean), and |k_j|^2 comes from pass 1: no key is read twice
+//                                   by CUDA cores
 // The finalize step (softmax of a, max-pool, lambda-mix) is the one the CUDA-core path uses.
 //
-// A CTA owns one (head, slice of key tiles).  Warps 0-3 read the logits from tensor memory, warps 4-7 read the
-// key tile from shared memory (norms, column sums, dot with the mean key), warp 8 streams key tiles through a
+// A CTA owns one (head, slice of key tiles).  Warps 0-3 read the logits from tensor memory, warps 4-7 (pass 1
+// only) read the key tile from shared memory (norms, column sums), warp 8 streams key tiles through a
 // 4-stage TMA ring and issues the MMAs into a 2-deep tensor-memory ring.  Keys are read from HBM once: the
 // second pass finds them in L2 for the cache sizes of the paper (a head is a few MB).
 // Sums are fixed-order: results are bit-reproducible from run to run.  Every mbarrier wait is bounded.
@@ -35,10 +39,9 @@ constexpr int kThreads = 288;  // warps 0-3 logits, warps 4-7 key vectors, warp 
 constexpr int kNQ = fc::kScoreTcMaxQueries;  // queries of pass 2 (MMA N), zero-padded
 
 struct TcSmem {
-  uint64_t q_full, k_full[kRing], k_free[kRing], s_full[2], s_free[2];
+  uint64_t q_full, q_patched, k_full[kRing], k_free[kRing], s_full[2], s_free[2];
   uint32_t tmem_base, abort;
   float inv_s[2][kKeys];   // 1 / |k| of the current tile's keys (double-buffered by tile parity)
-  float vec_s[128];        // pass 2: mean normalised key
   float lse_s[kNQ];        // pass 2: log2-domain log-sum-exp per query
   float red_m[2][4], red_l[2][4];
   float colsum_s[16][128];  // pass 1: per row-group column sums at the end of the slice
@@ -71,14 +74,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   TcSmem* sh = (TcSmem*)(smem + (1 + kRing) * kTileBytes);
   volatile uint32_t* abort = &sh->abort;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int hk = blockIdx.y, slice = blockIdx.x;
+  // Pass 2 walks heads, slices and tiles in the reverse of pass 1's order: what pass 1 read last is still in L2.
+  const int hk = PASS == 1 ? blockIdx.y : gridDim.y - 1 - blockIdx.y;
+  const int slice = PASS == 1 ? blockIdx.x : gridDim.x - 1 - blockIdx.x;
   const int t0 = slice * g.tiles_per_slice, t1 = min(g.n_tiles, t0 + g.tiles_per_slice), n = t1 - t0;
+  // i-th tile of this CTA
+  auto tile_of = [&](int i) { return PASS == 1 ? t0 + i : t1 - 1 - i; };
 
   if (tid == 0) {
     mbar_init(smem_u32(&sh->q_full), 1);
+    mbar_init(smem_u32(&sh->q_patched), 128);
     for (int s = 0; s < kRing; ++s) {
       mbar_init(smem_u32(&sh->k_full[s]), 1);
-      mbar_init(smem_u32(&sh->k_free[s]), 5);  // the MMA's commit and warps 4-7
+      mbar_init(smem_u32(&sh->k_free[s]), PASS == 1 ? 5 : 1);  // the MMA's commit and, in pass 1, warps 4-7
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&sh->s_full[b]), 1);
@@ -90,7 +98,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     tma_prefetch_desc(&tmap_k);
   }
   if (PASS == 2) {
-    if (tid < D) sh->vec_s[tid] = g.mean_key[hk * D + tid];
     if (tid < kNQ) sh->lse_s[tid] = g.lse2[hk * kNQ + tid];
   }
   if (warp == 0) {
@@ -105,18 +112,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   if (warp == 8) {
     // ---------------------------------------------------------------- copies and MMAs (one thread)
     if (lane == 0 && n > 0) {
-      auto load_k = [&](int i) {  // tile t0 + i into stage i % kRing
+      auto load_k = [&](int i) {  // i-th tile of the CTA into stage i % kRing
         const int st = i % kRing;
         const uint32_t bar = smem_u32(&sh->k_full[st]);
         mbar_expect_tx(bar, kTileBytes);
         for (int x = 0; x < kAtoms; ++x)
-          tma_load_3d(smem_u32(k_tiles + st * kTileBytes + x * kAtomBytes), &tmap_k, bar, x * 64, (t0 + i) * kKeys, hk);
+          tma_load_3d(smem_u32(k_tiles + st * kTileBytes + x * kAtomBytes), &tmap_k, bar, x * 64, tile_of(i) * kKeys, hk);
       };
       mbar_expect_tx(smem_u32(&sh->q_full), kTileBytes);
       for (int x = 0; x < kAtoms; ++x)
         tma_load_3d(smem_u32(q_tile + x * kAtomBytes), &tmap_q, smem_u32(&sh->q_full), x * 64, 0, hk);
       for (int i = 0; i < min(n, kRing - 1); ++i) load_k(i);
       mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
+      if (PASS == 2) mbar_wait_bounded(smem_u32(&sh->q_patched), 0, abort);
       const uint64_t dq = smem_desc_sw128(smem_u32(q_tile), 16, 1024);
       constexpr uint32_t kIdesc = PASS == 1 ? idesc_bf16_f32(128, kKeys, false, false) : idesc_bf16_f32(kKeys, kNQ, false, false);
       for (int i = 0; i < n; ++i) {
@@ -157,7 +165,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
         if (!warp_ok) continue;
-        const int cols_valid = min(kKeys, g.L_k - (t0 + i) * kKeys);
+        const int cols_valid = min(kKeys, g.L_k - tile_of(i) * kKeys);
         if (cols_valid < kKeys) {
 #pragma unroll
           for (int c = 0; c < kKeys; ++c)
@@ -191,9 +199,28 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       }
       if (row_ok) g.ml_part[((int64_t)hk * g.n_slices + slice) * kNQ + q] = make_float2(m, l);
     } else {
-      const float inv_nq = 1.f / (float)g.L_q;
+      // The mean key joins the queries as rows kNQ-2 (bf16 high part) and kNQ-1 (low part) of the Q tile, which
+      // the copy zero-filled: generic-proxy writes, made visible to the tensor cores by the proxy fence.
+      mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
+      if (tid < D) {
+        const float mk = g.mean_key[hk * D + tid];
+        const __nv_bfloat16 hi = __float2bfloat16_rn(mk), lo = __float2bfloat16_rn(mk - __bfloat162float(hi));
+        const int c = tid >> 3, x = c >> 3, cc = c & 7, e = tid & 7;
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+          const int r = kNQ - 2 + part;
+          *reinterpret_cast<__nv_bfloat16*>(q_tile + x * kAtomBytes + r * 128 + ((cc ^ (r & 7)) << 4) + e * 2) = part ? lo : hi;
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      mbar_arrive(smem_u32(&sh->q_patched));
+      const float inv_nq = 1.f / (float)g.L_q, inv_lk = 1.f / (float)g.L_k;
       for (int i = 0; i < n; ++i) {
         const int b = i & 1;
+        const int tile_id = tile_of(i), j = tile_id * kKeys + tid;  // this thread's key
+        const bool valid = j < g.L_k;
+        const int64_t o = (int64_t)hk * g.L_k + j;
+        const float n2 = valid && g.accum_phase != 1 ? g.norm2[o] : 0.f;  // in flight while the logits arrive
         mbar_wait_bounded(smem_u32(&sh->s_full[b]), (i >> 1) & 1, abort);
         tc_fence_after();
         uint32_t sv[kNQ];
@@ -201,14 +228,12 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
-        const int j = (t0 + i) * kKeys + tid;  // this thread's key
-        float mass = 0.f;
+        float ms[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int q = 0; q < kNQ; ++q)
-          if (q < g.L_q) mass += ex2(fmaf(__uint_as_float(sv[q]), g.scale_log2, -sh->lse_s[q]));
-        mass *= inv_nq;
-        if (j < g.L_k) {
-          const int64_t o = (int64_t)hk * g.L_k + j;
+        for (int q = 0; q < kNQ - 2; ++q)
+          if (q < g.L_q) ms[q & 3] += ex2(fmaf(__uint_as_float(sv[q]), g.scale_log2, -sh->lse_s[q]));
+        const float mass = ((ms[0] + ms[1]) + (ms[2] + ms[3])) * inv_nq;
+        if (valid) {
           if (g.accum_phase == 1) {
             g.imp_accum[o] += mass;
           } else if (g.accum_phase == 2) {
@@ -219,12 +244,43 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             g.imp_out[o] = mass;
           }
         }
+        if (g.accum_phase == 1) continue;
+        float a = -INFINITY;
+        if (valid) {
+          const float dot = __uint_as_float(sv[kNQ - 2]) + __uint_as_float(sv[kNQ - 1]);
+          const float inv = 1.f / fmaxf(sqrtf(n2), 1e-12f);
+          a = dot * inv - (n2 * inv * inv) * inv_lk;
+          g.a_out[o] = a;
+        }
+        // softmax statistics (max, sum of exp) of a over the tile, fixed order
+        float m = a;
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, w));
+        float l = valid ? expf(a - m) : 0.f;
+#pragma unroll
+        for (int w = 16; w > 0; w >>= 1) l += __shfl_xor_sync(0xffffffffu, l, w);
+        if (lane == 0) {
+          sh->red_m[i & 1][warp] = m;
+          sh->red_l[i & 1][warp] = l;
+        }
+        named_barrier_128();
+        if (tid == 0) {
+          m = sh->red_m[i & 1][0];
+          l = sh->red_l[i & 1][0];
+          for (int w = 1; w < 4; ++w) {
+            const float m2 = sh->red_m[i & 1][w], l2 = sh->red_l[i & 1][w];
+            const float mn = fmaxf(m, m2);
+            l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
+            m = mn;
+          }
+          g.a_partial[hk * g.n_tiles + tile_id] = make_float2(m, l);
+        }
       }
     }
-  } else {
+  } else if (PASS == 1) {
     // ---------------------------------------------------------------- key vectors out of shared memory
     const int u = tid - 128;  // 0..127
-    if (PASS == 1) {
+    {
       // column sums of the normalised keys: this thread owns 16-byte chunk `c` of the rows r = rg (mod kGroups)
       constexpr int kGroups = 128 / kChunks;  // 8 for d = 128, 16 for d = 64
       const int c = u % kChunks, rg = u / kChunks;
@@ -235,7 +291,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const int st = i % kRing;
         mbar_wait_bounded(smem_u32(&sh->k_full[st]), (i / kRing) & 1, abort);
         const uint8_t* tile = k_tiles + st * kTileBytes;
-        float n2 = 0.f;
+        float n4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int cc = 0; cc < kChunks; ++cc) {
           const uint4 w = lds_key_chunk<D>(tile, u, cc);
@@ -243,10 +299,13 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
             const float lo = fc::bf16_lo(ww[e]), hi = fc::bf16_hi(ww[e]);
-            n2 = fmaf(lo, lo, n2);
-            n2 = fmaf(hi, hi, n2);
+            n4[e] = fmaf(lo, lo, n4[e]);
+            n4[e] = fmaf(hi, hi, n4[e]);
           }
         }
+        const float n2 = (n4[0] + n4[1]) + (n4[2] + n4[3]);
+        const int j = tile_of(i) * kKeys + u;
+        if (j < g.L_k) g.norm2[(int64_t)hk * g.L_k + j] = n2;  // pass 2 takes |k|^2 from here
         // rows past the end of the cache are zero-filled: 0 * (1 / 1e-12) = 0, they add nothing
         sh->inv_s[i & 1][u] = 1.f / fmaxf(sqrtf(n2), 1e-12f);
         named_barrier_128();
@@ -270,67 +329,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         float t = 0.f;
         for (int r = 0; r < kGroups; ++r) t += sh->colsum_s[r][u];
         g.colsum_part[((int64_t)hk * g.n_slices + slice) * D + u] = t;
-      }
-    } else {
-      for (int i = 0; i < n; ++i) {
-        const int st = i % kRing;
-        mbar_wait_bounded(smem_u32(&sh->k_full[st]), (i / kRing) & 1, abort);
-        const int tile_id = t0 + i, j = tile_id * kKeys + u;
-        const bool valid = j < g.L_k;
-        float a = -INFINITY;
-        if (g.accum_phase != 1) {
-          const uint8_t* tile = k_tiles + st * kTileBytes;
-          float n2 = 0.f, dot = 0.f;
-#pragma unroll
-          for (int cc = 0; cc < kChunks; ++cc) {
-            const uint4 w = lds_key_chunk<D>(tile, u, cc);
-            const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-            const float4 m0 = *reinterpret_cast<const float4*>(&sh->vec_s[cc * 8]);
-            const float4 m1 = *reinterpret_cast<const float4*>(&sh->vec_s[cc * 8 + 4]);
-            const float mk[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const float lo = fc::bf16_lo(ww[e]), hi = fc::bf16_hi(ww[e]);
-              n2 = fmaf(lo, lo, n2);
-              n2 = fmaf(hi, hi, n2);
-              dot = fmaf(mk[2 * e], lo, dot);
-              dot = fmaf(mk[2 * e + 1], hi, dot);
-            }
-          }
-          if (valid) {
-            const float inv = 1.f / fmaxf(sqrtf(n2), 1e-12f);
-            a = dot * inv - (n2 * inv * inv) / (float)g.L_k;
-            g.a_out[(int64_t)hk * g.L_k + j] = a;
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sh->k_free[st]));
-        if (g.accum_phase == 1) continue;
-        // softmax statistics of a over the tile, fixed tree
-        float m = a, l = valid ? 1.f : 0.f;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const float m2 = __shfl_down_sync(0xffffffffu, m, o), l2 = __shfl_down_sync(0xffffffffu, l, o);
-          const float mn = fmaxf(m, m2);
-          l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
-          m = mn;
-        }
-        if (lane == 0) {
-          sh->red_m[i & 1][warp - 4] = m;
-          sh->red_l[i & 1][warp - 4] = l;
-        }
-        named_barrier_128();
-        if (u == 0) {
-          m = sh->red_m[i & 1][0];
-          l = sh->red_l[i & 1][0];
-          for (int w = 1; w < 4; ++w) {
-            const float m2 = sh->red_m[i & 1][w], l2 = sh->red_l[i & 1][w];
-            const float mn = fmaxf(m, m2);
-            l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
-            m = mn;
-          }
-          g.a_partial[hk * g.n_tiles + tile_id] = make_float2(m, l);
-        }
       }
     }
   }
@@ -378,8 +376,8 @@ int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs g, int d, int64_t q_h
   int rc;
   if ((rc = make_tmap(ctx, &tq, Q, d, g.L_q, g.H, q_rs, g.H > 1 ? q_hs : q_rs * g.L_q)) != FC_OK) return rc;
   if ((rc = make_tmap(ctx, &tk, K, d, g.L_k, g.H, k_rs, g.H > 1 ? k_hs : k_rs * g.L_k)) != FC_OK) return rc;
-  // slices: about two CTAs per SM over all heads, at most kScoreTcMaxSlices per head
-  const int want = std::max(1, (2 * ctx->sm_count + g.H - 1) / g.H);
+  // slices: one CTA per SM over all heads (a single wave), at most kScoreTcMaxSlices per head
+  const int want = std::max(1, ctx->sm_count / g.H);
   g.n_slices = std::min(std::min(want, kScoreTcMaxSlices), g.n_tiles);
   g.tiles_per_slice = (g.n_tiles + g.n_slices - 1) / g.n_slices;
   g.n_slices = (g.n_tiles + g.tiles_per_slice - 1) / g.tiles_per_slice;  // no empty slice

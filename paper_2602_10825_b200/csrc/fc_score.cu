@@ -356,7 +356,7 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
     a.H = g.H_kv; a.L_q = g.L_q; a.L_k = g.L_k; a.n_tiles = g.n_tiles; a.tiles_per_slice = 0; a.n_slices = 0;
     a.scale_log2 = g.scale * 1.4426950408889634f;
     a.accum_phase = accum_phase; a.n_steps = n_steps;
-    a.ml_part = w.tc_ml; a.colsum_part = w.tc_colsum; a.lse2 = w.tc_lse2; a.mean_key = w.mean_key; a.norm2 = w.tc_norm2;
+    a.ml_part = w.tc_ml; a.colsum_part = w.tc_colsum; a.norm2 = w.tc_norm2;
     a.imp_accum = imp_accum; a.imp_out = imp ? imp : w.imp_tmp; a.a_out = w.a; a.a_partial = w.a_partial;
     a.status = status;
     rc = fc::score_tc_run(ctx, st, a, g.d, g.q_hs, g.q_rs, g.k_hs, g.k_rs, Q_obs, K_cand);

@@ -17,8 +17,6 @@ struct ScoreTcArgs {
   int accum_phase, n_steps;
   float2* ml_part;     // [H, n_slices, 64] running (max, sum) of pass 1, log2 domain
   float* colsum_part;  // [H, n_slices, d] sums of normalised keys
-  float* lse2;         // [H, 64]
-  float* mean_key;     // [H, d]
   float* norm2;        // [H, L_k] squared l2 norm of every key (pass 1 -> pass 2)
   float* imp_accum;    // caller's accumulator or NULL
   float* imp_out;      // [H, L_k]
@@ -27,7 +25,7 @@ struct ScoreTcArgs {
   uint32_t* status;
 };
 
-// pass 1, merge, pass 2; the caller runs the finalize kernel afterwards (unless accum_phase == 1)
+// pass 1, pass 2; the caller runs the finalize kernel afterwards (unless accum_phase == 1)
 int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs args, int d, int64_t q_hs, int64_t q_rs, int64_t k_hs,
                  int64_t k_rs, const void* Q, const void* K);
 

@@ -8,7 +8,8 @@
 //   pass 1  S[query, key] = Q K^T   one query row per thread: running (max, sum) over the keys of the slice;
 //                                   the same pass adds up the l2-normalised keys (the mean key of the
 //                                   paper's efficiency appendix)
-//   merge   per head: slices' (max, sum) -> log-sum-exp per query; slice sums -> mean normalised key
+//           (every pass-2 CTA first merges its head's slice results: (max, sum) -> log-sum-exp per query, slice
+//           sums -> mean normalised key)
 //   pass 2  S[key, query] = K Q^T   one key row per thread: attention mass of the key; redundancy logit
 //                                   a_j = meankey . khat_j - |khat_j|^2 / L_k and its per-tile softmax statistics.
 //                                   The mean key rides along as two more query rows (its bf16 high and low
@@ -97,8 +98,20 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
   }
-  if (PASS == 2) {
-    if (tid < kNQ) sh->lse_s[tid] = g.lse2[hk * kNQ + tid];
+  if (PASS == 2 && tid < kNQ) {
+    // log-sum-exp of query `tid` over the whole head: pass 1's per-slice (max, sum) pairs, merged in slice order
+    float lse = 0.f;
+    if (tid < g.L_q) {
+      float m = -INFINITY, l = 0.f;
+      for (int s = 0; s < g.n_slices; ++s) {
+        const float2 p = g.ml_part[((int64_t)hk * g.n_slices + s) * kNQ + tid];
+        const float mn = fmaxf(m, p.x);
+        l = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * exp2f(p.x - mn));
+        m = mn;
+      }
+      lse = m + log2f(l);
+    }
+    sh->lse_s[tid] = lse;
   }
   if (warp == 0) {
     tmem_alloc(smem_u32(&sh->tmem_base), 2 * kCols);
@@ -203,7 +216,9 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       // the copy zero-filled: generic-proxy writes, made visible to the tensor cores by the proxy fence.
       mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
       if (tid < D) {
-        const float mk = g.mean_key[hk * D + tid];
+        float mk = 0.f;  // mean normalised key: pass 1's per-slice column sums, added in slice order
+        for (int s = 0; s < g.n_slices; ++s) mk += g.colsum_part[((int64_t)hk * g.n_slices + s) * D + tid];
+        mk /= (float)g.L_k;
         const __nv_bfloat16 hi = __float2bfloat16_rn(mk), lo = __float2bfloat16_rn(mk - __bfloat162float(hi));
         const int c = tid >> 3, x = c >> 3, cc = c & 7, e = tid & 7;
 #pragma unroll
@@ -342,30 +357,6 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   if (warp == 0) tmem_dealloc(tmem, 2 * kCols);
 }
 
-// per head: slices' (max, sum) -> log2-domain log-sum-exp per query; slices' column sums -> mean normalised key
-__global__ void score_tc_merge_kernel(const fc::ScoreTcArgs g, int d) {
-  const int hk = blockIdx.x, t = threadIdx.x;
-  if (t < kNQ) {
-    float lse = 0.f;
-    if (t < g.L_q) {
-      float m = -INFINITY, l = 0.f;
-      for (int s = 0; s < g.n_slices; ++s) {
-        const float2 p = g.ml_part[((int64_t)hk * g.n_slices + s) * kNQ + t];
-        const float mn = fmaxf(m, p.x);
-        l = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * exp2f(p.x - mn));
-        m = mn;
-      }
-      lse = m + log2f(l);
-    }
-    g.lse2[hk * kNQ + t] = lse;
-  }
-  if (t < d) {
-    float acc = 0.f;
-    for (int s = 0; s < g.n_slices; ++s) acc += g.colsum_part[((int64_t)hk * g.n_slices + s) * d + t];
-    g.mean_key[hk * d + t] = acc / (float)g.L_k;
-  }
-}
-
 }  // namespace
 
 namespace fc {
@@ -390,8 +381,6 @@ int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs g, int d, int64_t q_h
     return FC_OK;
   };
   if ((rc = d == 128 ? launch(score_tc_kernel<128, 1>) : launch(score_tc_kernel<64, 1>)) != FC_OK) return rc;
-  score_tc_merge_kernel<<<g.H, 128, 0, st>>>(g, d);
-  FC_LAUNCH_CHECK("score_tc_merge_kernel");
   return d == 128 ? launch(score_tc_kernel<128, 2>) : launch(score_tc_kernel<64, 2>);
 }
 

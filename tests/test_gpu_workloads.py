@@ -1,0 +1,143 @@
+"""The streaming and the sweep workloads end to end on the GPU against the CPU oracle, at sizes the oracle
+finishes in seconds: same chunk counts, step counts, thresholds and key statistics as the full configurations,
+fewer heads and shorter chunks (still several 128-token tiles with ragged tails).
+
+Bars as elsewhere: decisions and kept indices bit-exact (the selection is fed the same fp32 scores on both
+sides), compacted rows byte-exact, bf16 attention within max-abs 1e-2 / relative-L2 1e-2, scores within 1e-4
+of the row maximum.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    import paper_2602_10825_b200 as fc
+    from paper_2602_10825_b200 import build as fc_build
+    fc_build.build()
+    c = fc.Context(0)
+    yield c
+    c.close()
+
+
+def i32(x):
+    return torch.as_tensor(np.asarray(x), dtype=torch.int32).cuda()
+
+
+def _check_attention(got, want, atol=1e-2, rel=1e-2):
+    assert np.abs(got - want).max() <= atol
+    assert np.linalg.norm(got - want) <= rel * np.linalg.norm(want)
+
+
+def test_streaming_generation_with_compression_after_every_chunk(ctx):
+    # config 4 in small: chunks generated one after another, each denoised for S steps while attending to
+    # [history | itself]; the importance is accumulated over the chunk's steps; after the chunk the history is
+    # scored, the top B kept and compacted.  The first chunks fill the budget (identity), the rest compress.
+    full = wl.CONFIGS["streaming_bf16"]
+    H, d, n_c, B, n_chunks, S = 2, full.d, 328, 900, 7, full.n_steps
+    keys = list(wl.ar1_keys(H, n_chunks, n_c, d, seed=full.seed, sigma=full.sigma))
+    hist_K = torch.empty((H, 0, d), dtype=torch.bfloat16)
+    hist_V = torch.empty((H, 0, d), dtype=torch.bfloat16)
+    n_compress = 0
+    for c in range(n_chunks):
+        K_c = keys[c]
+        V_c = wl.normal((H, n_c, d), 7000 + c, full.sigma, torch.bfloat16)
+        K_all, V_all = torch.cat([hist_K, K_c], 1).contiguous(), torch.cat([hist_V, V_c], 1).contiguous()
+        L_hist, L_all = hist_K.shape[1], hist_K.shape[1] + n_c
+        q_off, vis = np.array([0, n_c], np.int32), np.array([L_all], np.int32)
+        slo = np.array([0, L_hist, L_all] if L_hist else [0, L_all], np.int32)
+        spo = np.array([0, L_hist] if L_hist else [0], np.int32)
+        acc_g = torch.zeros((H, L_all), device="cuda")
+        acc_o = np.zeros((H, L_all), np.float64)
+        Kg, Vg = K_all.cuda(), V_all.cuda()
+        for s in range(S):
+            Q = wl.normal((H, n_c, d), 8000 + 10 * c + s, full.sigma, torch.bfloat16)
+            O = torch.zeros((H, n_c, d), dtype=torch.bfloat16, device="cuda")
+            ctx.chunk_attention(Q.cuda(), Kg, Vg, q_off, vis, slo, spo, i32([0]), i32([1]), O)
+            rows = wl.sample_rows(wl.Workload("x", "bf16", H=H, d=d, W=1, n_c=n_c, B=0, L_k=0, seed=c), 6, s)
+            O_want, _ = oracle.chunk_attention(wl.bits(Q), wl.bits(K_all), wl.bits(V_all), q_off, vis, slo, spo, [0],
+                                               sample_rows=rows)
+            _check_attention(O.double().cpu().numpy()[:, rows], O_want)
+            Q_obs = Q[:, n_c - full.L_q_obs:].contiguous()
+            phase = 2 if s == S - 1 else 1
+            want = oracle.kv_score(wl.bits(Q_obs), wl.bits(K_all), lambda_=full.lam, pool_k=full.pool_k,
+                                   imp_accum=acc_o, accum_phase=phase, n_steps=S)
+            got = ctx.kv_score(Q_obs.cuda(), Kg, lambda_=full.lam, pool_k=full.pool_k, imp_accum=acc_g,
+                               accum_phase=phase, n_steps=S)
+        torch.cuda.synchronize()
+        score = got["score"].cpu().numpy()
+        assert np.abs(score - want["score"]).max() <= 1e-4 * np.abs(want["score"]).max()
+        sel = ctx.kv_select_compact(got["score"], B, Kg, Vg)
+        want_sel = oracle.kv_select_compact(score, B, wl.bits(K_all), wl.bits(V_all))
+        torch.cuda.synchronize()
+        assert np.array_equal(sel["kept_idx"].cpu().numpy(), want_sel["kept_idx"])
+        assert np.array_equal(wl.bits(sel["K_dst"].cpu()), want_sel["K_dst"])
+        assert np.array_equal(wl.bits(sel["V_dst"].cpu()), want_sel["V_dst"])
+        if L_all <= B:  # fill phase: nothing is dropped
+            assert np.array_equal(want_sel["kept_idx"], np.tile(np.arange(L_all, dtype=np.int32), (H, 1)))
+        else:
+            n_compress += 1
+            assert sel["kept_idx"].shape[1] == B
+        hist_K, hist_V = sel["K_dst"].cpu(), sel["V_dst"].cpu()
+    assert n_compress >= 4
+
+
+@pytest.mark.parametrize("eps", [0.05, 0.1, 0.2])
+def test_denoising_sweep_decisions_and_attention_of_the_active_chunks(ctx, eps):
+    # config 5 in small: 16 chunks, 30 steps, the change indicator shrinking from step to step so that the
+    # share of recomputed chunks falls from all of them to a few; decisions bit-exact at every step, attention
+    # of exactly the active chunks checked at the first step, in the middle and at the end.
+    full = wl.CONFIGS["sweep_bf16"]
+    w = wl.Workload("sweep_small", "bf16", H=2, d=full.d, W=full.W, n_c=200, B=456, L_k=656, seed=full.seed,
+                    sigma=full.sigma, D=256)
+    n_el = w.n_c * w.hidden
+    off = np.arange(w.W + 1, dtype=np.int64) * n_el
+    targets = wl.sweep_targets(full.n_steps, w.W, full.seed).numpy()
+    Q, K, V = wl.qkv(w)
+    q_off, vis, slo, spo = wl.prefix_layout(w)
+    Qg, Kg, Vg = Q.cuda(), K.cuda(), V.cuda()
+    O0 = wl.normal((w.H, w.window_rows, w.d), 77, 1.0, torch.bfloat16)
+    acc_o = np.zeros(w.W, np.float32)
+    acc_g = torch.zeros(w.W, device="cuda")
+    fractions = []
+    min_margin = np.inf
+    for s in range(full.n_steps):
+        step = np.full(w.W, s, np.int32)
+        target = targets[s].copy()
+        for _ in range(8):  # guard band: a draw that lands a chunk on the threshold is nudged away from it
+            cur, prev = wl.indicator_pair(w.W, n_el, target, 5000 + s)
+            want = oracle.chunk_decide(wl.bits(cur), wl.bits(prev), off, step, 1, eps, acc_o)
+            margin = np.abs(acc_o + want["l1rel"] - eps)
+            if s == 0 or margin.min() > 1e-3 * eps:
+                break
+            target[margin <= 1e-3 * eps] *= 1.03
+        if s >= 1:
+            min_margin = min(min_margin, float(margin.min()))
+        got = ctx.chunk_decide(cur.cuda(), prev.cuda(), off, i32(step), 1, eps, acc_g)
+        torch.cuda.synchronize()
+        assert got["recompute"].cpu().numpy().tolist() == want["recompute"].tolist(), f"step {s}"
+        assert got["active_ids"].cpu().numpy()[:want["n_active"]].tolist() == want["active_ids"].tolist()
+        acc_o = want["acc"]
+        active = want["active_ids"].tolist()
+        fractions.append(len(active) / w.W)
+        if s in (0, full.n_steps // 2, full.n_steps - 1):
+            O = O0.cuda().clone()
+            ctx.chunk_attention(Qg, Kg, Vg, q_off, vis, slo, spo, got["active_ids"], got["n_active"], O)
+            torch.cuda.synchronize()
+            rows = wl.sample_rows(w, 16, s)
+            rows = rows[np.isin(rows // w.n_c, active)]
+            if len(rows):
+                O_want, _ = oracle.chunk_attention(wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, slo, spo, active,
+                                                   sample_rows=rows)
+                _check_attention(O.double().cpu().numpy()[:, rows], O_want)
+            for c in range(w.W):  # chunks served from cache keep their outputs bit for bit
+                if c not in active:
+                    assert torch.equal(O[:, q_off[c]:q_off[c + 1]].cpu(), O0[:, q_off[c]:q_off[c + 1]])
+    assert min_margin > 1e-3 * eps, f"a step came within {min_margin} of eps; change the seed"
+    assert fractions[0] == 1.0 and fractions[-1] <= 0.5 and min(fractions) < max(fractions)

@@ -38,7 +38,7 @@ constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
 // of every 32 columns, this many (the last ones) take the polynomial exponential
 #ifndef FC_ATTN_EMU_COLS
-#define FC_ATTN_EMU_COLS 8
+#define FC_ATTN_EMU_COLS 0
 #endif
 constexpr int kEmuCols = FC_ATTN_EMU_COLS;
 // Registers per thread after the split: softmax warpgroups / the warpgroup of the copy and MMA warps.
@@ -63,6 +63,18 @@ constexpr bool kStagger = FC_ATTN_STAGGER != 0;
 #define FC_ATTN_PACE_CHUNK 0
 #endif
 constexpr int kPaceChunk = FC_ATTN_PACE_CHUNK;
+// exponentiate against the running reference before the tile's maximum is known (see the softmax loop)
+#ifndef FC_ATTN_SPECULATE
+#define FC_ATTN_SPECULATE 1
+#endif
+constexpr bool kSpeculate = FC_ATTN_SPECULATE != 0;
+// Option: two exponentials per special-function instruction (argument rounded to half precision, ex2 on the
+// packed pair).  Accuracy is unchanged (P is rounded to bf16 anyway), but the two extra conversions per pair cost
+// more issue slots than the special-function unit gains: measured slower on B200, so off.
+#ifndef FC_ATTN_EXP_F16X2
+#define FC_ATTN_EXP_F16X2 0
+#endif
+constexpr bool kExpF16x2 = FC_ATTN_EXP_F16X2 != 0;
 #define FC_STR2(x) #x
 #define FC_STR(x) FC_STR2(x)
 
@@ -83,6 +95,15 @@ struct WsSmem {
 struct Item {
   int h, hk, c, row0, n_vis;
 };
+
+// 2^x for a pair through the packed half-precision ex2: x0 in the low half.  Arguments below -65504 are clamped
+// by the conversion's saturation to -inf -> 0.
+__device__ __forceinline__ void ex2_f16x2(float x0, float x1, float& y0, float& y1) {
+  uint32_t h;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h) : "f"(x1), "f"(x0));
+  asm("ex2.approx.f16x2 %0, %0;" : "+r"(h));
+  asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\ncvt.f32.f16 %0, lo;\ncvt.f32.f16 %1, hi;\n}\n" : "=f"(y0), "=f"(y1) : "r"(h));
+}
 
 // 2^x for a pair, x <= 8, on the fma pipe: n = round(x) through the 1.5 * 2^23 shift, 2^(x-n) as a cubic
 // on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16 rounding of P), then n added to the exponent
@@ -107,11 +128,14 @@ __device__ __forceinline__ void ex2_poly2(float x0, float x1, float& y0, float& 
 }
 
 // P = 2^(S * scale - m) for one row of a 128-column tile, written back over S as bf16; returns the row sum.
-template <bool kAllEx2>
+// With kWithMax the raw row maximum of the tile is computed on the side (into `raw_max`): the caller used the
+// reference it already had and checks afterwards whether the tile's maximum allows that.
+template <bool kAllEx2, bool kWithMax>
 __device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s,
-                                          volatile uint32_t* half_flag, uint32_t half_value) {
+                                          volatile uint32_t* half_flag, uint32_t half_value, float& raw_max) {
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t sum2[2] = {0ull, 0ull};
+  float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
   constexpr int kEmuPairs = kAllEx2 ? 0 : kEmuCols / 2;
 #pragma unroll
   for (int q2 = 0; q2 < kBN / 32; ++q2) {
@@ -122,8 +146,12 @@ __device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale
                               sc2, nm2);
       float x0, x1, p0, p1;
       unpack2(x, x0, x1);
+      if (kWithMax)
+        mx[i & 3] = max3(mx[i & 3], __uint_as_float(sv[q2 * 32 + 2 * i]), __uint_as_float(sv[q2 * 32 + 2 * i + 1]));
       if (i >= 16 - kEmuPairs) {
         ex2_poly2(x0, x1, p0, p1);
+      } else if (kExpF16x2 && !kAllEx2) {
+        ex2_f16x2(x0, x1, p0, p1);
       } else {
         p0 = ex2(x0);
         p1 = ex2(x1);
@@ -134,6 +162,7 @@ __device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale
     tmem_st16(t_s + q2 * 16, pk);
     if (q2 == kPaceChunk && half_flag) *half_flag = half_value;  // this far through the tile
   }
+  if (kWithMax) raw_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
   float a, b, c, d;
   unpack2(sum2[0], a, b);
   unpack2(sum2[1], c, d);
@@ -414,27 +443,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           tc_fence_after();
           uint32_t sv[kBN];
           tmem_ld128_wait(t_s, sv);
-          if (cols_valid < kBN) {
-#pragma unroll
-            for (int i = 0; i < kBN; ++i)
-              if (i >= cols_valid) sv[i] = 0xff800000u;  // -inf
-          }
-          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-          for (int i = 0; i < kBN; i += 8) {
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4)
-              mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
-          }
-          const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
-          // lazy reference update: move only when the maximum grew by more than the threshold
-          float alpha = 1.f;
-          const bool move = tile_max > m + kRescaleThreshold;  // always true on the first tile (m = -inf)
-          if (move) {
-            alpha = ex2(m - tile_max);
-            m = tile_max;
-          }
-          if (j > 0 && __any_sync(0xffffffffu, move)) {
+          auto rescale_o = [&](float alpha) {
 #pragma unroll
             for (int q4 = 0; q4 < D / 32; ++q4) {
               uint32_t r[32];
@@ -443,10 +452,58 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
               for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
               tmem_st32(t_o + q4 * 32, r);
             }
+          };
+          float alpha = 1.f, row_sum, raw_max = 0.f;
+          if (kSpeculate && j > 0 && cols_valid == kBN) {
+            // Common case: the reference maximum of the row does not move (it moves only when a tile exceeds it by
+            // 2^8).  So exponentiate against the reference at once, without looking for the tile's maximum first.
+            // A row whose tile sum stays below 2^8 cannot hold a term above 2^8; only if some row of the warp
+            // exceeds that is the maximum computed, and the tile redone for the rows that have to move.
+            row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, half_flag, kv + 1, raw_max);
+            if (__any_sync(0xffffffffu, !(row_sum <= 256.f))) {  // 2^kRescaleThreshold; also catches inf / NaN
+              float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+              for (int i = 0; i < kBN; i += 8) {
+#pragma unroll
+                for (int c4 = 0; c4 < 4; ++c4)
+                  mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
+              }
+              const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
+              const bool move = tile_max > m + kRescaleThreshold;
+              if (__any_sync(0xffffffffu, move)) {
+                if (move) {
+                  alpha = ex2(m - tile_max);
+                  m = tile_max;
+                }
+                rescale_o(alpha);
+                row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, nullptr, 0, raw_max);
+              }
+            }
+          } else {
+            if (cols_valid < kBN) {
+#pragma unroll
+              for (int i = 0; i < kBN; ++i)
+                if (i >= cols_valid) sv[i] = 0xff800000u;  // -inf
+            }
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int i = 0; i < kBN; i += 8) {
+#pragma unroll
+              for (int c4 = 0; c4 < 4; ++c4)
+                mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
+            }
+            const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
+            // lazy reference update: move only when the maximum grew by more than the threshold
+            const bool move = tile_max > m + kRescaleThreshold;  // always true on the first tile (m = -inf)
+            if (move) {
+              alpha = ex2(m - tile_max);
+              m = tile_max;
+            }
+            if (j > 0 && __any_sync(0xffffffffu, move)) rescale_o(alpha);
+            // a ragged tile takes ex2 everywhere so that its masked columns give exactly 0
+            row_sum = cols_valid < kBN ? exp_tile<true, false>(sv, scale_log2, m, t_s, half_flag, kv + 1, raw_max)
+                                       : exp_tile<false, false>(sv, scale_log2, m, t_s, half_flag, kv + 1, raw_max);
           }
-          // a ragged tile takes ex2 everywhere so that its masked columns give exactly 0
-          const float row_sum = cols_valid < kBN ? exp_tile<true>(sv, scale_log2, m, t_s, half_flag, kv + 1)
-                                                 : exp_tile<false>(sv, scale_log2, m, t_s, half_flag, kv + 1);
           l = l * alpha + row_sum;
           tmem_wait_st();
           tc_fence_before();

@@ -131,7 +131,7 @@ class DeviceStep:
         self.n_kept = torch.empty(1, dtype=torch.int32, device=device)
         self.K_dst = torch.empty(H, self.n_keep, d, dtype=dt, device=device)
         self.V_dst = torch.empty(H, self.n_keep, d, dtype=dt, device=device)
-        self.launches_per_step = 2 + 1 + 3 + 3  # decide, attention, score (2 passes, finalize), select+compact
+        self.launches_per_step = 2 + 1 + 3 + 2  # decide, attention, score (2 passes, finalize), select, gather
 
     def decide(self):
         self.ctx.chunk_decide(self.cur, self.prev, self.chunk_off, self.chunk_step, self.w.warmup_m, self.w.eps,

@@ -2,8 +2,9 @@
 // retention of the selected K/V rows (Sec. 3.3).
 //
 // Selection: one 1024-thread block per head.  Scores become order-preserving 32-bit keys (NaN
-// ranks as -inf, -0 as +0) held in shared memory when they fit; a 4-pass, 8-bit-digit radix
-// select finds the key T of the B-th largest score and how many keys exceed it; one ordered
+// ranks as -inf, -0 as +0) held in shared memory when they fit; an 8-bit-digit radix select over
+// the bits in which the head's keys differ (at most 4 passes) finds the key T of the B-th largest
+// score and how many keys exceed it; one ordered
 // compaction then keeps every key above T plus the lowest-index keys equal to T, so the kept
 // set is exactly the first B elements of the total order (score descending, index ascending),
 // written in ascending index order.  Integer work only: bit-exact.
@@ -27,61 +28,122 @@ __device__ __forceinline__ uint32_t score_key(float s, bool& is_nan) {
 template <bool kSmemKeys>
 __global__ void __launch_bounds__(kSelThreads)
 select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __restrict__ kept_idx,
-                   uint32_t* __restrict__ status) {
+                   int32_t* __restrict__ n_kept, uint32_t* __restrict__ status) {
   extern __shared__ uint32_t smem_keys[];
-  __shared__ uint32_t hist[256];
+  __shared__ uint32_t hist[4][256];  // four copies, one per quarter of the warps, to spread the atomics
   __shared__ uint32_t sh_prefix, sh_remaining, sh_nan;
   const int h = blockIdx.x, tid = threadIdx.x;
   const float* s = score + (size_t)h * L_k;
   int32_t* out = kept_idx + (size_t)h * B;  // B <= L_k here (the identity case is handled apart)
 
   if (tid == 0) sh_nan = 0;
+  if (tid == 0 && h == 0 && n_kept) *n_kept = B;
   __syncthreads();
   bool any_nan = false;
-  if (kSmemKeys) {
-    for (int j = tid; j < L_k; j += kSelThreads) {
-      bool n;
-      smem_keys[j] = score_key(s[j], n);
-      any_nan |= n;
+  const int lane = tid & 31, warp = tid >> 5;
+  // Keys, and their range.  The scores of a head sit in a narrow band, so their keys share the leading bits;
+  // digits taken from the raw keys would send almost every key of the first passes to one histogram bin (and
+  // one shared-memory atomic at a time).  The select therefore works on key - min(key), which keeps the order,
+  // and starts at the highest bit in which the keys of this head differ.
+  uint32_t kmin = 0xffffffffu, kmax = 0;
+  for (int j0 = tid; j0 < L_k; j0 += 4 * kSelThreads) {
+    float v[4];  // four loads in flight per thread
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + u * kSelThreads;
+      v[u] = j < L_k ? s[j] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + u * kSelThreads;
+      if (j < L_k) {
+        bool n;
+        const uint32_t k = score_key(v[u], n);
+        any_nan |= n;
+        if (kSmemKeys) smem_keys[j] = k;
+        kmin = min(kmin, k);
+        kmax = max(kmax, k);
+      }
     }
   }
-  auto key_at = [&](int j) -> uint32_t {
-    if (kSmemKeys) return smem_keys[j];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+    kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+  }
+  __shared__ uint32_t red_min[kSelThreads / 32], red_max[kSelThreads / 32];
+  if (lane == 0) {
+    red_min[warp] = kmin;
+    red_max[warp] = kmax;
+  }
+  __syncthreads();
+#pragma unroll 1
+  for (int w = 0; w < kSelThreads / 32; ++w) {
+    kmin = min(kmin, red_min[w]);
+    kmax = max(kmax, red_max[w]);
+  }
+  const uint32_t base = kmin;
+  const int n_bits = 32 - __clz(kmax - kmin);  // 0 when all keys are equal
+  auto key_at = [&](int j) -> uint32_t {  // key relative to the head's minimum
+    if (kSmemKeys) return smem_keys[j] - base;
     bool n;
-    uint32_t k = score_key(s[j], n);
-    any_nan |= n;
-    return k;
+    return score_key(s[j], n) - base;
   };
 
-  // Radix select, most significant digit first.  Invariant: the B-th largest key has the bits
-  // of `prefix` in the digits already fixed, and `remaining` of the keys with that prefix
+  // Radix select, most significant digit first, 8 bits at a time over the n_bits that vary.  Invariant: the
+  // B-th largest key has the bits of `prefix` above bit `hi`, and `remaining` of the keys with that prefix
   // (counted from the largest) are still to be taken.
-  uint32_t prefix = 0, prefix_mask = 0, remaining = (uint32_t)B;
-  for (int shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
+  uint32_t prefix = 0, remaining = (uint32_t)B;
+  for (int hi = n_bits; hi > 0;) {
+    const int lo = max(hi - 8, 0);
+    const uint32_t digit_mask = (1u << (hi - lo)) - 1u;
+    hist[tid >> 8][tid & 255] = 0;
     __syncthreads();
     for (int j = tid; j < L_k; j += kSelThreads) {
       const uint32_t k = key_at(j);
-      if ((k & prefix_mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1u);
+      const bool candidate = hi >= 32 || (k >> hi) == (prefix >> hi);
+      if (candidate) atomicAdd(&hist[warp & 3][(k >> lo) & digit_mask], 1u);
     }
     __syncthreads();
-    if (tid == 0) {
-      uint32_t rem = remaining;
-      int digit = 255;
-      for (; digit > 0; --digit) {
-        if (hist[digit] >= rem) break;
-        rem -= hist[digit];
+    if (tid < 32) {
+      // digits from 255 downwards, eight per lane; the digit of the B-th largest key is where the running
+      // count first reaches `remaining`
+      uint32_t c[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int bin = 255 - (tid * 8 + i);
+        c[i] = (hist[0][bin] + hist[1][bin]) + (hist[2][bin] + hist[3][bin]);
+        tot += c[i];
       }
-      sh_prefix = prefix | ((uint32_t)digit << shift);
-      sh_remaining = rem;
+      uint32_t inc = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
+        if (tid >= o) inc += v;
+      }
+      const uint32_t exc = inc - tot;
+      if (exc < remaining && remaining <= inc) {
+        uint32_t rem = remaining - exc;
+        int digit = 255 - tid * 8;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (c[i] >= rem) {
+            digit = 255 - (tid * 8 + i);
+            break;
+          }
+          rem -= c[i];
+        }
+        sh_prefix = prefix | ((uint32_t)digit << lo);
+        sh_remaining = rem;
+      }
     }
     __syncthreads();
     prefix = sh_prefix;
     remaining = sh_remaining;
-    prefix_mask |= 255u << shift;
+    hi = lo;
     __syncthreads();
   }
-  const uint32_t T = prefix;           // key of the B-th largest score
+  const uint32_t T = prefix;           // key (relative to the minimum) of the B-th largest score
   const uint32_t need_eq = remaining;  // how many keys equal to T are kept (lowest indices)
 
   // Ordered compaction: thread t owns the contiguous index range [t*per, (t+1)*per).
@@ -96,7 +158,6 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __r
   // exclusive block scan of the packed pair (eq in the high half, gt in the low half)
   uint32_t packed = (n_eq << 16) | n_gt;  // per-thread counts < 65536 (L_k/1024 items per thread)
   uint32_t incl = packed;
-  const int lane = tid & 31, warp = tid >> 5;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
@@ -132,8 +193,10 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __r
 }
 
 __global__ void select_identity_kernel(int32_t* __restrict__ kept_idx, int n_heads, int L_k,
-                                       const float* __restrict__ score, uint32_t* __restrict__ status) {
+                                       const float* __restrict__ score, int32_t* __restrict__ n_kept,
+                                       uint32_t* __restrict__ status) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i == 0 && n_kept) *n_kept = L_k;
   if (i >= (int64_t)n_heads * L_k) return;
   kept_idx[i] = (int32_t)(i % L_k);
   if (status) {
@@ -142,7 +205,6 @@ __global__ void select_identity_kernel(int32_t* __restrict__ kept_idx, int n_hea
   }
 }
 
-__global__ void write_count_kernel(int32_t* n_kept, int32_t v) { *n_kept = v; }
 
 // Row gather.  The copy of one head is a flat list of 16-byte pieces: piece p of the head
 // belongs to kept row p / pieces_per_row.  A block moves kUnroll * blockDim pieces of K and of V;
@@ -189,7 +251,7 @@ gather_rows_kernel(const uint8_t* __restrict__ K_src, const uint8_t* __restrict_
     }
 }
 
-constexpr size_t kStaticSelSmem = 256 * 4 + 3 * (kSelThreads / 32) * 4 + 64;
+constexpr size_t kStaticSelSmem = 4 * 256 * 4 + 4 * (kSelThreads / 32) * 4 + 64;  // histograms, per-warp scratch, scalars
 
 }  // namespace
 
@@ -225,22 +287,18 @@ extern "C" int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* scor
   const int n_keep = B < L_k ? B : L_k;
   if (B >= L_k) {
     const int64_t n = (int64_t)n_heads * L_k;
-    select_identity_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kept_idx, n_heads, L_k, score, status);
+    select_identity_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kept_idx, n_heads, L_k, score, n_kept, status);
     FC_LAUNCH_CHECK("select_identity_kernel");
   } else {
     const size_t key_bytes = (size_t)L_k * 4;
     if (key_bytes + kStaticSelSmem + 1024 <= (size_t)ctx->smem_optin) {
       FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
-      select_topb_kernel<true><<<n_heads, kSelThreads, key_bytes, st>>>(score, L_k, B, kept_idx, status);
+      select_topb_kernel<true><<<n_heads, kSelThreads, key_bytes, st>>>(score, L_k, B, kept_idx, n_kept, status);
     } else {
-      select_topb_kernel<false><<<n_heads, kSelThreads, 0, st>>>(score, L_k, B, kept_idx, status);
+      select_topb_kernel<false><<<n_heads, kSelThreads, 0, st>>>(score, L_k, B, kept_idx, n_kept, status);
     }
     FC_LAUNCH_CHECK("select_topb_kernel");
-  }
-  if (n_kept) {
-    write_count_kernel<<<1, 1, 0, st>>>(n_kept, n_keep);
-    FC_LAUNCH_CHECK("write_count_kernel");
   }
   if (copy) {
     const int es = fc::elem_size(dtype);

@@ -31,6 +31,13 @@ sys.path.insert(0, ROOT)
 import workloads as wl  # noqa: E402
 
 NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 8000.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, from the ncu captures summarised under profiles/
+# (taken with the kernels as they are in this tree; set an entry to None when its kernel changes)
+NCU_TRAFFIC = {
+    ("single_step_bf16", "attention_ws_kernel"): 650.1e6 + 85.4e6,
+    ("single_step_bf16", "gather_rows_kernel"): 206.1e6 + 153.6e6,
+    ("cached_step_bf16", "gather_rows_kernel"): 231.8e6 + 180.0e6,
+}
 FALLBACK = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
@@ -163,6 +170,21 @@ class DeviceStep:
 
 def attention_flops(w, active):
     return w.attention_flops(active)
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a few per-rank timings over all ranks (the slowest rank sets the job's time).
+    `dist` is torch.distributed or None for a single process."""
+    if dist is None:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(world, flops_per_rank_step, ms_per_step):
+    """Whole-job TFLOP/s of `world` replicas that each do `flops_per_rank_step` per step (weak scaling)."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
 
 
 def time_device(step, steps, warmup, barrier):
@@ -321,21 +343,17 @@ def main():
     if not args.no_e2e:
         e2e_steps = max(2, min(args.steps // 4, 40))
         e2e_ms, h2d, d2h = time_e2e(step, e2e_steps, args.warmup, barrier)
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms / e2e_steps if not args.no_e2e else 0.0], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t[0])
-        e2e_step_ms = float(t[1])
-    else:
-        e2e_step_ms = e2e_ms / e2e_steps if not args.no_e2e else 0.0
+    total_ms, e2e_step_ms = max_over_ranks([total_ms, e2e_ms / e2e_steps if not args.no_e2e else 0.0], dist, device)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         ms_per_step = total_ms / args.steps
-        value = world * flops / (ms_per_step * 1e-3) / 1e12
+        value = job_throughput(world, flops, ms_per_step)
         attn_tflops = flops / (stage_ms["attention"] * 1e-3) / 1e12
         compact_bytes = 4 * step.n_keep * w.d * 2 * w.H
         compact_gbs = compact_bytes / (stage_ms["select_compact"] * 1e-3) / 1e9
+        score_gbs = step.L_k * w.d * 2 * w.H / (stage_ms["score"] * 1e-3) / 1e9
+        decide_gbs = 2 * step.cur.numel() * 2 / (stage_ms["decide"] * 1e-3) / 1e9
         line = {
             "metric": "chunk_attn_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -347,23 +365,33 @@ def main():
                        "parallelism": "replicas" if world > 1 else "single"},
             "stages_ms": stage_ms,
             "roofline": {"bound": "tensor", "achieved": attn_tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": attn_tflops / peaks["bf16_tflops"], "traffic": None, "kernel": "attention_ws_kernel",
+                         "frac": attn_tflops / peaks["bf16_tflops"],
+                         "traffic": NCU_TRAFFIC.get((w.name, "attention_ws_kernel")), "kernel": "attention_ws_kernel",
                          "peak_kind": peak_kind + " burst", "frac_of_nominal": attn_tflops / NOMINAL["bf16_tflops"],
                          "frac_of_sustained": attn_tflops / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])},
             "roofline_compact": {"bound": "hbm", "achieved": compact_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                                 "frac": compact_gbs / peaks["hbm_gbs"], "traffic": None,
+                                 "frac": compact_gbs / peaks["hbm_gbs"],
+                                 "traffic": NCU_TRAFFIC.get((w.name, "gather_rows_kernel")),
                                  "kernel": "select + gather_rows_kernel (whole fc_kv_select_compact call)",
                                  "peak_kind": peak_kind, "frac_of_nominal": compact_gbs / NOMINAL["hbm_gbs"]},
+            "roofline_score": {"bound": "hbm", "achieved": score_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                               "frac": score_gbs / peaks["hbm_gbs"], "traffic": None,
+                               "kernel": "score_tc_kernel passes 1 and 2 + score_finalize_kernel (whole fc_kv_score call); "
+                                         "algorithmic bytes = the candidate keys once", "peak_kind": peak_kind},
+            "roofline_decide": {"bound": "hbm", "achieved": decide_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                "frac": decide_gbs / peaks["hbm_gbs"], "traffic": None,
+                                "kernel": "decide_partial_kernel + decide_finalize_kernel (whole fc_chunk_decide call)",
+                                "peak_kind": peak_kind},
             "clocks": clocks, "device_status": status,
             "gpu_launches": step.launches_per_step * args.steps,
         }
         if not args.no_e2e:
-            line["e2e"] = {"value": world * flops / (e2e_step_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+            line["e2e"] = {"value": job_throughput(world, flops, e2e_step_ms), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_step_ms}
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
-            dt, fl, cores, desc = oracle_sample(w, 0, 768)
+            dt, fl, cores, desc = oracle_sample(w, 0, 1536)
             line["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": cores, "kind": "oracle",
                                     "sample": desc + f" ({dt:.1f} s)"}
         print(json.dumps(line))

@@ -1,7 +1,7 @@
 // fc_kv_select_compact: per-head top-B of the selection score (text after Eq. 12) and the
 // retention of the selected K/V rows (Sec. 3.3).
 //
-// Selection: one 1024-thread block per head.  Scores become order-preserving 32-bit keys (NaN
+// Selection: one cluster of four 1024-thread blocks per head, each holding a quarter of the head's keys.  Scores become order-preserving 32-bit keys (NaN
 // ranks as -inf, -0 as +0) held in shared memory when they fit; an 8-bit-digit radix select over
 // the bits in which the head's keys differ (at most 4 passes) finds the key T of the B-th largest
 // score and how many keys exceed it; one ordered
@@ -11,6 +11,8 @@
 //
 // Compaction: a separate streaming kernel moves whole rows with 16-byte accesses, several
 // independent loads in flight per thread; rows that were dropped are never read.
+#include <cooperative_groups.h>
+
 #include "fc_common.cuh"
 
 namespace {
@@ -25,41 +27,57 @@ __device__ __forceinline__ uint32_t score_key(float s, bool& is_nan) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // larger float <=> larger key
 }
 
+// One cluster of kSelCluster CTAs per head; CTA r of the cluster owns the contiguous index range
+// [r * chunk, (r + 1) * chunk) of the head.  The CTAs exchange their partial results (minimum / maximum, digit
+// histograms, counts of kept keys) by reading each other's shared memory.
+constexpr int kSelCluster = 4;
+
+struct SelShared {
+  uint32_t hist[4][256];   // four copies, one per quarter of the warps, to spread the atomics
+  uint32_t hist_cta[256];  // this CTA's histogram of the current digit (read by the other CTAs)
+  uint32_t red_min[kSelThreads / 32], red_max[kSelThreads / 32];
+  uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32];
+  uint32_t cta_min, cta_max, cta_gt, cta_eq;  // read by the other CTAs
+  uint32_t prefix, remaining, nan;
+};
+
 template <bool kSmemKeys>
 __global__ void __launch_bounds__(kSelThreads)
-select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __restrict__ kept_idx,
+select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, int32_t* __restrict__ kept_idx,
                    int32_t* __restrict__ n_kept, uint32_t* __restrict__ status) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ uint32_t smem_keys[];
-  __shared__ uint32_t hist[4][256];  // four copies, one per quarter of the warps, to spread the atomics
-  __shared__ uint32_t sh_prefix, sh_remaining, sh_nan;
-  const int h = blockIdx.x, tid = threadIdx.x;
-  const float* s = score + (size_t)h * L_k;
+  __shared__ SelShared sh;
+  const int rank = (int)cluster.block_rank(), h = blockIdx.x / kSelCluster, tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  const int begin = min(rank * chunk, L_k), n = min(begin + chunk, L_k) - begin;  // this CTA's keys: begin + [0, n)
+  const float* s = score + (size_t)h * L_k + begin;
   int32_t* out = kept_idx + (size_t)h * B;  // B <= L_k here (the identity case is handled apart)
 
-  if (tid == 0) sh_nan = 0;
-  if (tid == 0 && h == 0 && n_kept) *n_kept = B;
+  if (tid == 0) sh.nan = 0;
+  if (tid == 0 && blockIdx.x == 0 && n_kept) *n_kept = B;
   __syncthreads();
   bool any_nan = false;
-  const int lane = tid & 31, warp = tid >> 5;
   // Keys, and their range.  The scores of a head sit in a narrow band, so their keys share the leading bits;
   // digits taken from the raw keys would send almost every key of the first passes to one histogram bin (and
   // one shared-memory atomic at a time).  The select therefore works on key - min(key), which keeps the order,
   // and starts at the highest bit in which the keys of this head differ.
   uint32_t kmin = 0xffffffffu, kmax = 0;
-  for (int j0 = tid; j0 < L_k; j0 += 4 * kSelThreads) {
+  for (int j0 = tid; j0 < n; j0 += 4 * kSelThreads) {
     float v[4];  // four loads in flight per thread
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int j = j0 + u * kSelThreads;
-      v[u] = j < L_k ? s[j] : 0.f;
+      v[u] = j < n ? s[j] : 0.f;
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int j = j0 + u * kSelThreads;
-      if (j < L_k) {
-        bool n;
-        const uint32_t k = score_key(v[u], n);
-        any_nan |= n;
+      if (j < n) {
+        bool nn;
+        const uint32_t k = score_key(v[u], nn);
+        any_nan |= nn;
         if (kSmemKeys) smem_keys[j] = k;
         kmin = min(kmin, k);
         kmax = max(kmax, k);
@@ -71,50 +89,66 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __r
     kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
     kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
   }
-  __shared__ uint32_t red_min[kSelThreads / 32], red_max[kSelThreads / 32];
   if (lane == 0) {
-    red_min[warp] = kmin;
-    red_max[warp] = kmax;
+    sh.red_min[warp] = kmin;
+    sh.red_max[warp] = kmax;
   }
   __syncthreads();
-#pragma unroll 1
-  for (int w = 0; w < kSelThreads / 32; ++w) {
-    kmin = min(kmin, red_min[w]);
-    kmax = max(kmax, red_max[w]);
+  if (tid == 0) {
+    for (int w = 0; w < kSelThreads / 32; ++w) {
+      kmin = min(kmin, sh.red_min[w]);
+      kmax = max(kmax, sh.red_max[w]);
+    }
+    sh.cta_min = kmin;
+    sh.cta_max = kmax;
+  }
+  cluster.sync();
+  kmin = 0xffffffffu;
+  kmax = 0;
+  for (int q = 0; q < kSelCluster; ++q) {
+    const SelShared* other = cluster.map_shared_rank(&sh, q);
+    kmin = min(kmin, other->cta_min);
+    kmax = max(kmax, other->cta_max);
   }
   const uint32_t base = kmin;
-  const int n_bits = 32 - __clz(kmax - kmin);  // 0 when all keys are equal
-  auto key_at = [&](int j) -> uint32_t {  // key relative to the head's minimum
+  const int n_bits = kmax >= kmin ? 32 - __clz(kmax - kmin) : 0;  // 0 when all keys are equal
+  auto key_at = [&](int j) -> uint32_t {  // key relative to the head's minimum; j is local to this CTA
     if (kSmemKeys) return smem_keys[j] - base;
-    bool n;
-    return score_key(s[j], n) - base;
+    bool nn;
+    return score_key(s[j], nn) - base;
   };
 
   // Radix select, most significant digit first, 8 bits at a time over the n_bits that vary.  Invariant: the
   // B-th largest key has the bits of `prefix` above bit `hi`, and `remaining` of the keys with that prefix
-  // (counted from the largest) are still to be taken.
+  // (counted from the largest) are still to be taken.  Every CTA adds up all CTAs' histograms and takes the
+  // same decision.
   uint32_t prefix = 0, remaining = (uint32_t)B;
   for (int hi = n_bits; hi > 0;) {
     const int lo = max(hi - 8, 0);
     const uint32_t digit_mask = (1u << (hi - lo)) - 1u;
-    hist[tid >> 8][tid & 255] = 0;
+    sh.hist[tid >> 8][tid & 255] = 0;
     __syncthreads();
-    for (int j = tid; j < L_k; j += kSelThreads) {
+    for (int j = tid; j < n; j += kSelThreads) {
       const uint32_t k = key_at(j);
       const bool candidate = hi >= 32 || (k >> hi) == (prefix >> hi);
-      if (candidate) atomicAdd(&hist[warp & 3][(k >> lo) & digit_mask], 1u);
+      if (candidate) atomicAdd(&sh.hist[warp & 3][(k >> lo) & digit_mask], 1u);
     }
     __syncthreads();
+    if (tid < 256) sh.hist_cta[tid] = (sh.hist[0][tid] + sh.hist[1][tid]) + (sh.hist[2][tid] + sh.hist[3][tid]);
+    cluster.sync();
     if (tid < 32) {
       // digits from 255 downwards, eight per lane; the digit of the B-th largest key is where the running
       // count first reaches `remaining`
       uint32_t c[8], tot = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int bin = 255 - (tid * 8 + i);
-        c[i] = (hist[0][bin] + hist[1][bin]) + (hist[2][bin] + hist[3][bin]);
-        tot += c[i];
+      for (int i = 0; i < 8; ++i) c[i] = 0;
+      for (int q = 0; q < kSelCluster; ++q) {
+        const SelShared* other = cluster.map_shared_rank(&sh, q);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) c[i] += other->hist_cta[255 - (tid * 8 + i)];
       }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) tot += c[i];
       uint32_t inc = tot;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -133,22 +167,21 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __r
           }
           rem -= c[i];
         }
-        sh_prefix = prefix | ((uint32_t)digit << lo);
-        sh_remaining = rem;
+        sh.prefix = prefix | ((uint32_t)digit << lo);
+        sh.remaining = rem;
       }
     }
-    __syncthreads();
-    prefix = sh_prefix;
-    remaining = sh_remaining;
+    cluster.sync();  // every CTA has read the histograms before the next pass clears them
+    prefix = sh.prefix;
+    remaining = sh.remaining;
     hi = lo;
-    __syncthreads();
   }
   const uint32_t T = prefix;           // key (relative to the minimum) of the B-th largest score
   const uint32_t need_eq = remaining;  // how many keys equal to T are kept (lowest indices)
 
-  // Ordered compaction: thread t owns the contiguous index range [t*per, (t+1)*per).
-  const int per = (L_k + kSelThreads - 1) / kSelThreads;
-  const int j0 = min(tid * per, L_k), j1 = min(j0 + per, L_k);
+  // Ordered compaction: thread t owns the contiguous local range [t*per, (t+1)*per).
+  const int per = (n + kSelThreads - 1) / kSelThreads;
+  const int j0 = min(tid * per, n), j1 = min(j0 + per, n);
   uint32_t n_gt = 0, n_eq = 0;
   for (int j = j0; j < j1; ++j) {
     const uint32_t k = key_at(j);
@@ -156,7 +189,7 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __r
     n_eq += k == T;
   }
   // exclusive block scan of the packed pair (eq in the high half, gt in the low half)
-  uint32_t packed = (n_eq << 16) | n_gt;  // per-thread counts < 65536 (L_k/1024 items per thread)
+  uint32_t packed = (n_eq << 16) | n_gt;  // per-thread counts < 65536 (at most L_k/1024 items per thread)
   uint32_t incl = packed;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -164,32 +197,41 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int32_t* __r
     if (lane >= o) incl += v;
   }
   // a warp's totals stay below 2^16 per half (L_k <= 2^20); block-level bases use full words
-  __shared__ uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32];
   if (lane == 31) {
-    warp_gt[warp] = incl & 0xffffu;
-    warp_eq[warp] = incl >> 16;
+    sh.warp_gt[warp] = incl & 0xffffu;
+    sh.warp_eq[warp] = incl >> 16;
   }
   __syncthreads();
   uint32_t base_gt = 0, base_eq = 0;
   for (int w = 0; w < warp; ++w) {
-    base_gt += warp_gt[w];
-    base_eq += warp_eq[w];
+    base_gt += sh.warp_gt[w];
+    base_eq += sh.warp_eq[w];
+  }
+  if (tid == kSelThreads - 1) {  // this CTA's totals, for the CTAs that own higher indices
+    sh.cta_gt = base_gt + (incl & 0xffffu);
+    sh.cta_eq = base_eq + (incl >> 16);
+  }
+  cluster.sync();
+  for (int q = 0; q < rank; ++q) {
+    const SelShared* other = cluster.map_shared_rank(&sh, q);
+    base_gt += other->cta_gt;
+    base_eq += other->cta_eq;
   }
   uint32_t gt_before = base_gt + (incl & 0xffffu) - n_gt;
   uint32_t eq_before = base_eq + (incl >> 16) - n_eq;
   for (int j = j0; j < j1; ++j) {
     const uint32_t k = key_at(j);
     if (k > T) {
-      out[gt_before + min(eq_before, need_eq)] = j;
+      out[gt_before + min(eq_before, need_eq)] = begin + j;
       ++gt_before;
     } else if (k == T) {
-      if (eq_before < need_eq) out[gt_before + eq_before] = j;
+      if (eq_before < need_eq) out[gt_before + eq_before] = begin + j;
       ++eq_before;
     }
   }
-  if (any_nan) sh_nan = 1;
-  __syncthreads();
-  if (tid == 0 && sh_nan && status) atomicOr(status, FC_DEV_NAN_SCORE);
+  if (any_nan) sh.nan = 1;
+  cluster.sync();  // no CTA leaves while another may still read its shared memory
+  if (tid == 0 && sh.nan && status) atomicOr(status, FC_DEV_NAN_SCORE);
 }
 
 __global__ void select_identity_kernel(int32_t* __restrict__ kept_idx, int n_heads, int L_k,
@@ -251,7 +293,6 @@ gather_rows_kernel(const uint8_t* __restrict__ K_src, const uint8_t* __restrict_
     }
 }
 
-constexpr size_t kStaticSelSmem = 4 * 256 * 4 + 4 * (kSelThreads / 32) * 4 + 64;  // histograms, per-warp scratch, scalars
 
 }  // namespace
 
@@ -290,13 +331,27 @@ extern "C" int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* scor
     select_identity_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kept_idx, n_heads, L_k, score, n_kept, status);
     FC_LAUNCH_CHECK("select_identity_kernel");
   } else {
-    const size_t key_bytes = (size_t)L_k * 4;
-    if (key_bytes + kStaticSelSmem + 1024 <= (size_t)ctx->smem_optin) {
+    const int chunk = (L_k + kSelCluster - 1) / kSelCluster;
+    const size_t key_bytes = (size_t)chunk * 4;
+    const bool smem_keys = key_bytes + sizeof(SelShared) + 1024 <= (size_t)ctx->smem_optin;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_heads * kSelCluster);
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = smem_keys ? key_bytes : 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = kSelCluster;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (smem_keys) {
       FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
-      select_topb_kernel<true><<<n_heads, kSelThreads, key_bytes, st>>>(score, L_k, B, kept_idx, n_kept, status);
+      FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<true>, score, L_k, B, chunk, kept_idx, n_kept, status));
     } else {
-      select_topb_kernel<false><<<n_heads, kSelThreads, 0, st>>>(score, L_k, B, kept_idx, n_kept, status);
+      FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<false>, score, L_k, B, chunk, kept_idx, n_kept, status));
     }
     FC_LAUNCH_CHECK("select_topb_kernel");
   }

@@ -206,6 +206,64 @@ def test_attention_bf16_tensor_core_small(ctx, impl, d):
     _attention_case(ctx, w2, [0, 1], impl=impl, atol=1e-2, rel_l2=1e-2)
 
 
+def _attention_custom(ctx, Q, K, V, q_off, vis, slo, spo, active, impl, O0=None):
+    H_q, R, d = Q.shape
+    O0 = wl.normal((H_q, R, d), 555, 1.0, torch.bfloat16) if O0 is None else O0
+    Og = dev(O0).clone()
+    lse_g = torch.full((H_q, R), float("nan"), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    W = len(q_off) - 1
+    ctx.chunk_attention(dev(Q), dev(K), dev(V), q_off, vis, slo, spo, i32(list(active) + [-1] * (W - len(active))),
+                        i32([len(active)]), Og, lse=lse_g, impl=impl, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    O_want, lse_want = oracle.chunk_attention(wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, slo, spo, active,
+                                              O_init=O0.double().numpy())
+    got = Og.double().cpu().numpy()
+    assert np.abs(got - O_want).max() <= 1e-2
+    assert np.linalg.norm(got - O_want) <= 1e-2 * max(np.linalg.norm(O_want), 1e-30)
+    rows = np.concatenate([np.arange(q_off[c], q_off[c + 1]) for c in active]) if len(active) else np.array([], int)
+    lg, lw = lse_g.double().cpu().numpy()[:, rows], lse_want[:, rows]
+    finite = np.isfinite(lw)
+    np.testing.assert_allclose(lg[finite], lw[finite], atol=2e-3)
+    assert np.array_equal(np.isneginf(lg), np.isneginf(lw))
+    return Og
+
+
+@pytest.mark.parametrize("impl", [2, 3])
+def test_attention_tensor_core_edge_cases(ctx, impl):
+    d = 128
+    # grouped query heads: 4 query heads on 2 key heads
+    Q = wl.normal((4, 300, d), 61, 0.5, torch.bfloat16)
+    K = wl.normal((2, 400, d), 62, 0.5, torch.bfloat16)
+    V = wl.normal((2, 400, d), 63, 0.5, torch.bfloat16)
+    q_off, vis = np.array([0, 100, 300], np.int32), np.array([200, 400], np.int32)
+    _attention_custom(ctx, Q, K, V, q_off, vis, np.array([0, 400], np.int32), np.array([0], np.int32), [0, 1], impl)
+    # a clean region scattered over ten physical segments in shuffled order, chunks of unequal length, one of
+    # them empty, visible lengths that are not monotone, a chunk that sees nothing (output 0, LSE -inf)
+    rng = np.random.default_rng(3)
+    seg_len = [37, 128, 1, 255, 64, 129, 90, 7, 300, 13]
+    order = rng.permutation(len(seg_len))
+    phys = np.zeros(len(seg_len), np.int64)
+    pos = 5
+    for s_ in order:  # lay the segments out in shuffled order with gaps between them
+        phys[s_] = pos
+        pos += seg_len[s_] + int(rng.integers(0, 9))
+    slo = np.concatenate([[0], np.cumsum(seg_len)]).astype(np.int32)
+    L_phys = pos + 3
+    Q = wl.normal((2, 700, d), 64, 0.5, torch.bfloat16)
+    K = wl.normal((2, L_phys, d), 65, 0.5, torch.bfloat16)
+    V = wl.normal((2, L_phys, d), 66, 0.5, torch.bfloat16)
+    q_off = np.array([0, 130, 130, 400, 401, 700], np.int32)  # chunk 1 is empty, chunk 3 has one row
+    vis = np.array([slo[-1], 50, 0, 700, 166], np.int32)
+    _attention_custom(ctx, Q, K, V, q_off, vis, slo, phys.astype(np.int32), [0, 1, 2, 3, 4], impl)
+    _attention_custom(ctx, Q, K, V, q_off, vis, slo, phys.astype(np.int32), [2, 3], impl)
+    # nothing active: nothing is written
+    O0 = wl.normal((2, 700, d), 67, 1.0, torch.bfloat16)
+    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, phys.astype(np.int32), [], impl, O0=O0)
+    assert torch.equal(Og.cpu(), O0)
+
+
 def test_attention_bf16_many_items_per_cta(ctx):
     # more work items than SMs, of very different lengths: exercises the device-side item queue
     w = wl.Workload("q", "bf16", H=40, d=128, W=6, n_c=520, B=300, L_k=820, seed=18, sigma=0.5)

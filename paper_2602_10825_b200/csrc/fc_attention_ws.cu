@@ -58,7 +58,8 @@ static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg 
 #define FC_ATTN_STAGGER 1
 #endif
 constexpr bool kStagger = FC_ATTN_STAGGER != 0;
-// the pacing flag of a tile is raised after this 32-column chunk of its exponentials (0..3)
+// the pacing flag of a tile is raised after this 32-column chunk of its exponentials (0..3), or when its softmax
+// starts (-1)
 #ifndef FC_ATTN_PACE_CHUNK
 #define FC_ATTN_PACE_CHUNK 0
 #endif
@@ -131,7 +132,7 @@ __device__ __forceinline__ void ex2_poly2(float x0, float x1, float& y0, float& 
 // With kWithMax the raw row maximum of the tile is computed on the side (into `raw_max`): the caller used the
 // reference it already had and checks afterwards whether the tile's maximum allows that.
 template <bool kAllEx2, bool kWithMax>
-__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s,
+__device__ __forceinline__ float exp_tile(uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s,
                                           volatile uint32_t* half_flag, uint32_t half_value, float& raw_max) {
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t sum2[2] = {0ull, 0ull};
@@ -160,7 +161,18 @@ __device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale
       pk[i] = cvt_bf16x2(p0, p1);
     }
     tmem_st16(t_s + q2 * 16, pk);
-    if (q2 == kPaceChunk && half_flag) *half_flag = half_value;  // this far through the tile
+    if (q2 == kPaceChunk) {
+      if (half_flag) *half_flag = half_value;  // this far through the tile
+      // The flag must go out now, not after the compiler has moved the rest of the tile's arithmetic in front
+      // of it: the next chunk's inputs pass through an empty volatile statement placed after the store.
+      if (q2 + 1 < kBN / 32) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 8)
+          asm volatile("" : "+r"(sv[(q2 + 1) * 32 + i]), "+r"(sv[(q2 + 1) * 32 + i + 1]), "+r"(sv[(q2 + 1) * 32 + i + 2]),
+                            "+r"(sv[(q2 + 1) * 32 + i + 3]), "+r"(sv[(q2 + 1) * 32 + i + 4]), "+r"(sv[(q2 + 1) * 32 + i + 5]),
+                            "+r"(sv[(q2 + 1) * 32 + i + 6]), "+r"(sv[(q2 + 1) * 32 + i + 7]));
+      }
+    }
   }
   if (kWithMax) raw_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
   float a, b, c, d;
@@ -443,6 +455,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           tc_fence_after();
           uint32_t sv[kBN];
           tmem_ld128_wait(t_s, sv);
+          if (kPaceChunk < 0 && half_flag) *half_flag = kv + 1;  // pacing flag as soon as the tile's softmax starts
           auto rescale_o = [&](float alpha) {
 #pragma unroll
             for (int q4 = 0; q4 < D / 32; ++q4) {

@@ -172,6 +172,46 @@ def attention_flops(w, active):
     return w.attention_flops(active)
 
 
+def run_sweep(step, thresholds, n_steps, peak_tflops):
+    """The denoising sweep: per threshold, `n_steps` consecutive steps whose per-chunk change indicator shrinks
+    from step to step (u * kappa_s, u ~ U(0,1), kappa_s geometric from 1 to 0.02), so the share of recomputed
+    chunks falls from all of them to a few.  Each step runs decide -> attention with the active list staying on
+    the device; per step the realised active fraction, the stage times and the attention roofline fraction."""
+    w, dev = step.w, step.device
+    n_el = w.n_c * w.hidden
+    g = torch.Generator(device=dev)
+    g.manual_seed(4242)
+    sign = (torch.randint(0, 2, (w.W, n_el), generator=g, device=dev, dtype=torch.int8) * 2 - 1)
+    prev = step.prev.view(w.W, n_el)
+    out = []
+    for eps in thresholds:
+        step.acc.zero_()
+        rows = []
+        for s in range(n_steps):
+            kappa = 0.02 ** (s / max(n_steps - 1, 1))
+            r = torch.rand(w.W, 1, generator=g, device=dev) * kappa
+            step.cur.view(w.W, n_el).copy_((prev.float() * (1 + r * sign)).to(prev.dtype))
+            step.chunk_step.fill_(s)
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            ev[0].record()
+            step.ctx.chunk_decide(step.cur, step.prev, step.chunk_off, step.chunk_step, 1, eps, step.acc,
+                                  l1rel=step.l1rel, recompute=step.recompute, active_ids=step.active_ids,
+                                  n_active=step.n_active, status=step.status)
+            ev[1].record()
+            step.attention()
+            ev[2].record()
+            torch.cuda.synchronize()
+            n_act = int(step.n_active.item())
+            active = step.active_ids[:n_act].cpu().tolist()
+            att_ms = ev[1].elapsed_time(ev[2])
+            tf = attention_flops(w, active) / (att_ms * 1e-3) / 1e12 if n_act else 0.0
+            rows.append({"step": s, "active_fraction": n_act / w.W, "decide_ms": ev[0].elapsed_time(ev[1]),
+                         "attention_ms": att_ms, "attention_tflops": tf, "frac": tf / peak_tflops})
+        out.append({"eps": eps, "steps": rows})
+    del sign
+    return out
+
+
 def max_over_ranks(values, dist, device):
     """Element-wise maximum of a few per-rank timings over all ranks (the slowest rank sets the job's time).
     `dist` is torch.distributed or None for a single process."""
@@ -297,6 +337,8 @@ def main():
     ap.add_argument("--impl", default="fc", choices=["fc", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="also run the 30-step denoising sweep at thresholds 0.05 / 0.1 / 0.2 and add it to the line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "fc" else args.warmup
     w = wl.CONFIGS[args.config]
@@ -388,6 +430,8 @@ def main():
         if not args.no_e2e:
             line["e2e"] = {"value": job_throughput(world, flops, e2e_step_ms), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_step_ms}
+        if args.sweep:
+            line["sweep"] = run_sweep(step, (0.05, 0.1, 0.2), 30, peaks["bf16_tflops"])
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()

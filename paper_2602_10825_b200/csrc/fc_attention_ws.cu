@@ -58,12 +58,11 @@ static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg 
 #define FC_ATTN_STAGGER 1
 #endif
 constexpr bool kStagger = FC_ATTN_STAGGER != 0;
-// the pacing flag of a tile is raised after this 32-column chunk of its exponentials (0..3), or when its softmax
-// starts (-1)
-#ifndef FC_ATTN_PACE_CHUNK
-#define FC_ATTN_PACE_CHUNK 0
+// clocks between the S groups of the two query tiles (see the pacing comment in the MMA threads)
+#ifndef FC_ATTN_PACE_DELAY
+#define FC_ATTN_PACE_DELAY 1100
 #endif
-constexpr int kPaceChunk = FC_ATTN_PACE_CHUNK;
+constexpr int kPaceDelay = FC_ATTN_PACE_DELAY;
 // exponentiate against the running reference before the tile's maximum is known (see the softmax loop)
 #ifndef FC_ATTN_SPECULATE
 #define FC_ATTN_SPECULATE 1
@@ -85,7 +84,8 @@ struct WsSmem {
   uint64_t s_full[2], p_ready[2], o_done[2];
   uint64_t it_full[2], it_empty[2];
   int32_t it_slot[2];
-  uint32_t half_done[2];  // per query tile: key tiles whose softmax its first warp has half finished (pacing hint)
+  uint32_t s_issued[2];   // per query tile: number of S groups its MMA thread has issued (pacing hint) ...
+  uint32_t s_clock[2];    // ... and the SM clock at the last of them
   uint32_t tmem_base;
   uint32_t abort;
   int32_t n_act, total_items;
@@ -95,6 +95,7 @@ struct WsSmem {
 
 struct Item {
   int h, hk, c, row0, n_vis;
+  bool b_valid;  // tile B has at least one row of the chunk (false for the ragged last item of a chunk)
 };
 
 // 2^x for a pair through the packed half-precision ex2: x0 in the low half.  Arguments below -65504 are clamped
@@ -132,8 +133,8 @@ __device__ __forceinline__ void ex2_poly2(float x0, float x1, float& y0, float& 
 // With kWithMax the raw row maximum of the tile is computed on the side (into `raw_max`): the caller used the
 // reference it already had and checks afterwards whether the tile's maximum allows that.
 template <bool kAllEx2, bool kWithMax>
-__device__ __forceinline__ float exp_tile(uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s,
-                                          volatile uint32_t* half_flag, uint32_t half_value, float& raw_max) {
+__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s,
+                                          float& raw_max) {
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t sum2[2] = {0ull, 0ull};
   float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -161,18 +162,6 @@ __device__ __forceinline__ float exp_tile(uint32_t (&sv)[kBN], float scale_log2,
       pk[i] = cvt_bf16x2(p0, p1);
     }
     tmem_st16(t_s + q2 * 16, pk);
-    if (q2 == kPaceChunk) {
-      if (half_flag) *half_flag = half_value;  // this far through the tile
-      // The flag must go out now, not after the compiler has moved the rest of the tile's arithmetic in front
-      // of it: the next chunk's inputs pass through an empty volatile statement placed after the store.
-      if (q2 + 1 < kBN / 32) {
-#pragma unroll
-        for (int i = 0; i < 32; i += 8)
-          asm volatile("" : "+r"(sv[(q2 + 1) * 32 + i]), "+r"(sv[(q2 + 1) * 32 + i + 1]), "+r"(sv[(q2 + 1) * 32 + i + 2]),
-                            "+r"(sv[(q2 + 1) * 32 + i + 3]), "+r"(sv[(q2 + 1) * 32 + i + 4]), "+r"(sv[(q2 + 1) * 32 + i + 5]),
-                            "+r"(sv[(q2 + 1) * 32 + i + 6]), "+r"(sv[(q2 + 1) * 32 + i + 7]));
-      }
-    }
   }
   if (kWithMax) raw_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
   float a, b, c, d;
@@ -227,7 +216,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     }
     mbar_fence_init();
     sh->abort = 0;
-    sh->half_done[0] = sh->half_done[1] = 0;
+    sh->s_issued[0] = sh->s_issued[1] = 0;
+    sh->s_clock[0] = sh->s_clock[1] = 0;
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
@@ -278,6 +268,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     it.row0 = g.q_row_off[it.c] + ((item - start) % pairs) * 2 * kBM;
     it.n_vis = g.vis[it.c];
     it.hk = it.h / g.group;
+    it.b_valid = it.row0 + kBM < g.q_row_off[it.c + 1];
     return it;
   };
   // consumer side of the item ring; -1 once the list is exhausted or the CTA has given up
@@ -387,19 +378,31 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const uint32_t b_vfull = smem_u32(&sh->v_full[0]), b_vempty = smem_u32(&sh->v_empty[0]);
     const uint32_t b_sfull = smem_u32(&sh->s_full[x]), b_pready = smem_u32(&sh->p_ready[x]);
     // Pacing.  Left alone, the two tiles fall into step: both softmaxes run together, sharing the special-
-    // function unit, and then both tiles' MMAs queue up behind each other.  So each S is issued only once the
-    // other tile's softmax is half way through its current key tile: S_B(j) after half of softmax A(j), S_A(j+1)
-    // after half of softmax B(j).  That keeps the two softmaxes about half a period apart, and one tile's MMAs
-    // run under the other tile's softmax.  It is only a delay: no data depends on it, and it gives up after 20 us.
+    // function unit, and then both tiles' MMAs queue up behind each other.  So each S is issued no earlier than
+    // kPaceDelay clocks after the other tile's S for its current key tile was issued: S_B(j) after S_A(j),
+    // S_A(j+1) after S_B(j).  That keeps the two softmaxes apart by a good part of a period, and one tile's MMAs
+    // run under the other tile's softmax.  The MMA threads time each other directly (their instruction streams
+    // are short and ordered); it is only a delay: no data depends on it, and it gives up after 20 us.
     auto pace = [&](uint32_t want) {
       if (!kStagger) return;
-      volatile uint32_t* other = &sh->half_done[x ^ 1];
-      if ((int32_t)(*other - want) >= 0) return;
+      volatile uint32_t* issued = &sh->s_issued[x ^ 1];
+      volatile uint32_t* clk = &sh->s_clock[x ^ 1];
       const uint64_t t0 = global_timer_ns();
-      while ((int32_t)(*other - want) < 0 && global_timer_ns() - t0 < 20000ull) {
+      while ((int32_t)(*issued - want) < 0) {
+        if (global_timer_ns() - t0 > 20000ull) return;
+      }
+      if (*issued != want) return;  // the other tile is further ahead than that: no need to wait
+      const uint32_t since = *clk;
+      while ((uint32_t)clock64() - since < (uint32_t)kPaceDelay) {
       }
     };
-    uint32_t kv = 0;
+    auto announce = [&](uint32_t n_issued, uint32_t back_date) {
+      *(volatile uint32_t*)&sh->s_clock[x] = (uint32_t)clock64() - back_date;
+      *(volatile uint32_t*)&sh->s_issued[x] = n_issued;
+    };
+    // Barrier phases are counted per use: tile B sits out the items in which it has no rows (the last item of a
+    // chunk whose length is not a multiple of 256), so its barriers see fewer phases than tile A's.
+    uint32_t kv = 0, uses = 0;
     for (uint32_t it_n = 0;; ++it_n) {
       const int slot = it_n & 1;
       mbar_wait_bounded(smem_u32(&sh->it_full[slot]), (it_n >> 1) & 1, abort);
@@ -410,7 +413,21 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       const int n_tiles = count_tiles(it);
       mbar_wait_bounded(smem_u32(&sh->q_full), it_n & 1, abort);
       tc_fence_after();
-      for (int j = 0; j < n_tiles; ++j, ++kv) {
+      if (x == 1 && !it.b_valid) {
+        // Nothing to compute for tile B.  Its arrivals on the ring barriers are still due, one stage at a time
+        // (waiting for the stage to be full keeps them in the right phase), and tile A still paces itself on it.
+        for (int j = 0; j < n_tiles; ++j, ++kv) {
+          const uint32_t st = kv & 1, ph = (kv >> 1) & 1;
+          mbar_wait_bounded(b_kfull + 8 * st, ph, abort);
+          mbar_arrive(b_kempty + 8 * st);
+          mbar_wait_bounded(b_vfull + 8 * st, ph, abort);
+          mbar_arrive(b_vempty + 8 * st);
+          if (kStagger) announce(kv + 1, kPaceDelay);
+        }
+        mbar_arrive(smem_u32(&sh->q_empty));
+        continue;
+      }
+      for (int j = 0; j < n_tiles; ++j, ++kv, ++uses) {
         const uint32_t st = kv & 1, ph = (kv >> 1) & 1;  // kStages == 2
         mbar_wait_bounded(b_kfull + 8 * st, ph, abort);
         pace(kv + x);
@@ -418,8 +435,9 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         issue_s(st);
         umma_commit(b_sfull);
         umma_commit(b_kempty + 8 * st);
+        if (kStagger) announce(kv + 1, 0);
         mbar_wait_bounded(b_vfull + 8 * st, ph, abort);
-        mbar_wait_bounded(b_pready, kv & 1, abort);
+        mbar_wait_bounded(b_pready, uses & 1, abort);
         tc_fence_after();
         issue_pv(st, j > 0);
         umma_commit(b_vempty + 8 * st);
@@ -438,24 +456,26 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const uint32_t t_o = tmem + lane_base + 256 + x * 128;
     const int r_in = (warp & 3) * 32 + lane;  // row inside the tile
     const float scale_log2 = g.scale * 1.4426950408889634f;
-    volatile uint32_t* half_flag = (kStagger && (warp & 3) == 0 && lane == 0) ? &sh->half_done[x] : nullptr;
-    uint32_t kv = 0;
+    uint32_t kv = 0, uses = 0, items = 0;  // tiles seen, tiles and items actually processed (barrier phases)
     for (uint32_t it_n = 0;; ++it_n) {
       const int item = next_item(it_n);
       if (item < 0) break;
       const Item it = decode(item);
+      if (x == 1 && !it.b_valid) {  // no row of the chunk in tile B: its MMA thread sits the item out too
+        kv += count_tiles(it);
+        continue;
+      }
       float m = -INFINITY, l = 0.f;
       int j = 0;
       for (int s = 0; s < g.n_seg; ++s) {
         const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
         if (seg_vis <= 0) break;
-        for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv, ++j) {
+        for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv, ++j, ++uses) {
           const int cols_valid = min(kBN, seg_vis - j0);
-          warp_wait(smem_u32(&sh->s_full[x]), kv & 1, abort);
+          warp_wait(smem_u32(&sh->s_full[x]), uses & 1, abort);
           tc_fence_after();
           uint32_t sv[kBN];
           tmem_ld128_wait(t_s, sv);
-          if (kPaceChunk < 0 && half_flag) *half_flag = kv + 1;  // pacing flag as soon as the tile's softmax starts
           auto rescale_o = [&](float alpha) {
 #pragma unroll
             for (int q4 = 0; q4 < D / 32; ++q4) {
@@ -472,7 +492,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             // 2^8).  So exponentiate against the reference at once, without looking for the tile's maximum first.
             // A row whose tile sum stays below 2^8 cannot hold a term above 2^8; only if some row of the warp
             // exceeds that is the maximum computed, and the tile redone for the rows that have to move.
-            row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, half_flag, kv + 1, raw_max);
+            row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, raw_max);
             if (__any_sync(0xffffffffu, !(row_sum <= 256.f))) {  // 2^kRescaleThreshold; also catches inf / NaN
               float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -489,7 +509,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                   m = tile_max;
                 }
                 rescale_o(alpha);
-                row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, nullptr, 0, raw_max);
+                row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, raw_max);
               }
             }
           } else {
@@ -514,8 +534,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             }
             if (j > 0 && __any_sync(0xffffffffu, move)) rescale_o(alpha);
             // a ragged tile takes ex2 everywhere so that its masked columns give exactly 0
-            row_sum = cols_valid < kBN ? exp_tile<true, false>(sv, scale_log2, m, t_s, half_flag, kv + 1, raw_max)
-                                       : exp_tile<false, false>(sv, scale_log2, m, t_s, half_flag, kv + 1, raw_max);
+            row_sum = cols_valid < kBN ? exp_tile<true, false>(sv, scale_log2, m, t_s, raw_max)
+                                       : exp_tile<false, false>(sv, scale_log2, m, t_s, raw_max);
           }
           l = l * alpha + row_sum;
           tmem_wait_st();
@@ -525,7 +545,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         }
       }
       // epilogue
-      warp_wait(smem_u32(&sh->o_done[x]), it_n & 1, abort);
+      warp_wait(smem_u32(&sh->o_done[x]), items & 1, abort);
+      ++items;
       tc_fence_after();
       const int row = it.row0 + x * kBM + r_in;
       const bool row_ok = row < g.q_row_off[it.c + 1];

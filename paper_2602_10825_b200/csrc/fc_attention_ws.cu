@@ -387,9 +387,11 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       if (!kStagger) return;
       volatile uint32_t* issued = &sh->s_issued[x ^ 1];
       volatile uint32_t* clk = &sh->s_clock[x ^ 1];
-      const uint64_t t0 = global_timer_ns();
-      while ((int32_t)(*issued - want) < 0) {
-        if (global_timer_ns() - t0 > 20000ull) return;
+      if ((int32_t)(*issued - want) < 0) {  // the global timer is slow to read: only when there is something to wait for
+        const uint64_t t0 = global_timer_ns();
+        while ((int32_t)(*issued - want) < 0) {
+          if (global_timer_ns() - t0 > 20000ull) return;
+        }
       }
       if (*issued != want) return;  // the other tile is further ahead than that: no need to wait
       const uint32_t since = *clk;

@@ -49,6 +49,7 @@ __device__ __forceinline__ void load_row(const T* __restrict__ row, float (&x)[D
 
 struct ScoreGeom {
   int H_q, H_kv, d, L_q, L_k, group, n_q, n_tiles;
+  int n_partials;  // softmax statistics of a per head handed to the finalize kernel (one per tile, or per warp of a tile)
   int64_t q_hs, q_rs, k_hs, k_rs;
   float scale, lambda;
   int pool_k;
@@ -214,35 +215,43 @@ score_pass2_kernel(const T* __restrict__ K, ScoreGeom g, const float* __restrict
   if (tid == 0) a_partial[hk * g.n_tiles + tile] = make_float2(m, l);
 }
 
-__global__ void __launch_bounds__(kTile)
+// One block finalises kFinKeys keys of a head: it first merges the head's partial softmax statistics of a (every
+// block of the head does, in the same fixed order), then writes redundancy, pooled importance and the score.
+constexpr int kFinThreads = 256, kFinKeys = 1024;
+
+__global__ void __launch_bounds__(kFinThreads)
 score_finalize_kernel(ScoreGeom g, const float* __restrict__ imp_in, const float* __restrict__ a_in,
                       const float2* __restrict__ a_partial, float* __restrict__ red_out,
                       float* __restrict__ score) {
-  __shared__ float sm_m[kTile / 32], sm_l[kTile / 32];
+  __shared__ float sm_m[kFinThreads / 32], sm_l[kFinThreads / 32];
   __shared__ float sh_m, sh_l;
-  const int hk = blockIdx.y, tile = blockIdx.x, tid = threadIdx.x;
+  const int hk = blockIdx.y, tid = threadIdx.x;
   float m = -INFINITY, l = 0.f;
-  for (int t = tid; t < g.n_tiles; t += kTile) {
-    const float2 p = a_partial[hk * g.n_tiles + t];
+  for (int t = tid; t < g.n_partials; t += kFinThreads) {
+    const float2 p = a_partial[hk * g.n_partials + t];
     const float mn = fmaxf(m, p.x);
     l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * expf(p.x - mn));
     m = mn;
   }
-  reduce_ml<kTile>(m, l, sm_m, sm_l);
+  reduce_ml<kFinThreads>(m, l, sm_m, sm_l);
   if (tid == 0) {
     sh_m = m;
     sh_l = l;
   }
   __syncthreads();
-  const int j = tile * kTile + tid;
-  if (j >= g.L_k) return;
   const int64_t base = (int64_t)hk * g.L_k;
-  const float red = expf(a_in[base + j] - sh_m) / sh_l;
   const int half = g.pool_k / 2;
-  float pooled = -INFINITY;
-  for (int u = max(j - half, 0); u <= min(j + half, g.L_k - 1); ++u) pooled = fmaxf(pooled, imp_in[base + u]);
-  if (red_out) red_out[base + j] = red;
-  score[base + j] = g.lambda * pooled - (1.f - g.lambda) * red;
+  const float inv_l = 1.f / sh_l;
+#pragma unroll
+  for (int i = 0; i < kFinKeys / kFinThreads; ++i) {
+    const int j = blockIdx.x * kFinKeys + i * kFinThreads + tid;
+    if (j >= g.L_k) break;
+    const float red = expf(a_in[base + j] - sh_m) * inv_l;
+    float pooled = -INFINITY;
+    for (int u = max(j - half, 0); u <= min(j + half, g.L_k - 1); ++u) pooled = fmaxf(pooled, imp_in[base + u]);
+    if (red_out) red_out[base + j] = red;
+    score[base + j] = g.lambda * pooled - (1.f - g.lambda) * red;
+  }
 }
 
 struct ScoreWs {
@@ -269,7 +278,7 @@ ScoreWs carve(const ScoreGeom& g, void* ws) {
   w.mean_key = (float*)take((size_t)g.H_kv * g.d * 4);
   w.a = (float*)take((size_t)g.H_kv * g.L_k * 4);
   w.imp_tmp = (float*)take((size_t)g.H_kv * g.L_k * 4);
-  w.a_partial = (float2*)take((size_t)g.H_kv * g.n_tiles * 8);
+  w.a_partial = (float2*)take((size_t)g.H_kv * g.n_tiles * 4 * 8);  // room for one entry per warp of a tile
   w.tc_ml = (float2*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * fc::kScoreTcMaxQueries * 8);
   w.tc_colsum = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * g.d * 4);
   w.tc_lse2 = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxQueries * 4);
@@ -288,6 +297,7 @@ int make_geom(const fc_score_desc* d, ScoreGeom& g) {
   g.n_q = g.group * d->L_q;
   if (g.n_q > 128) return FC_ERR_UNSUPPORTED;
   g.n_tiles = (d->L_k + kTile - 1) / kTile;
+  g.n_partials = g.n_tiles;
   g.q_hs = d->q_hs; g.q_rs = d->q_rs; g.k_hs = d->k_hs; g.k_rs = d->k_rs;
   g.scale = d->scale != 0.f ? d->scale : 1.f / sqrtf((float)d->d);
   g.lambda = d->lambda;
@@ -313,7 +323,7 @@ int run(cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, co
                                                    n_steps, imp_buf, w.a, w.a_partial);
   FC_LAUNCH_CHECK("score_pass2_kernel");
   if (phase != 1) {
-    score_finalize_kernel<<<grid, kTile, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
+    score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
     FC_LAUNCH_CHECK("score_finalize_kernel");
   }
   return FC_OK;
@@ -361,7 +371,8 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
     a.status = status;
     rc = fc::score_tc_run(ctx, st, a, g.d, g.q_hs, g.q_rs, g.k_hs, g.k_rs, Q_obs, K_cand);
     if (rc != FC_OK || accum_phase == 1) return rc;
-    score_finalize_kernel<<<dim3(g.n_tiles, g.H_kv), kTile, 0, st>>>(g, a.imp_out, w.a, w.a_partial, red, score);
+    g.n_partials = g.n_tiles * 4;  // the tensor-core pass leaves one entry per warp of a tile
+    score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, a.imp_out, w.a, w.a_partial, red, score);
     FC_LAUNCH_CHECK("score_finalize_kernel");
     return FC_OK;
   }

@@ -21,7 +21,7 @@ struct ScoreTcArgs {
   float* imp_accum;    // caller's accumulator or NULL
   float* imp_out;      // [H, L_k]
   float* a_out;        // [H, L_k] redundancy logits
-  float2* a_partial;   // [H, n_tiles] softmax statistics of a per 128-key tile
+  float2* a_partial;   // [H, n_tiles * 4] softmax statistics (max, sum of exp) of a per 32 keys (one warp of a tile)
   uint32_t* status;
 };
 

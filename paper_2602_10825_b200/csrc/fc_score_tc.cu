@@ -18,8 +18,9 @@
 //                                   by CUDA cores
 // The finalize step (softmax of a, max-pool, lambda-mix) is the one the CUDA-core path uses.
 //
-// A CTA owns one (head, slice of key tiles).  Warps 0-3 read the logits from tensor memory, warps 4-7 (pass 1
-// only) read the key tile from shared memory (norms, column sums), warp 8 streams key tiles through a
+// A CTA owns one (head, slice of key tiles).  Warps 0-3 read the logits from tensor memory; warps 4-7 read the
+// key tile from shared memory in pass 1 (norms, column sums) and are a second logit warpgroup in pass 2 (the
+// two take alternate tiles); warp 8 streams key tiles through a
 // 4-stage TMA ring and issues the MMAs into a 2-deep tensor-memory ring.  Keys are read from HBM once: the
 // second pass finds them in L2 for the cache sizes of the paper (a head is a few MB).
 // Sums are fixed-order: results are bit-reproducible from run to run.  Every mbarrier wait is bounded.
@@ -43,8 +44,7 @@ struct TcSmem {
   uint64_t q_full, q_patched, k_full[kRing], k_free[kRing], s_full[2], s_free[2];
   uint32_t tmem_base, abort;
   float inv_s[2][kKeys];   // 1 / |k| of the current tile's keys (double-buffered by tile parity)
-  float lse_s[kNQ];        // pass 2: log2-domain log-sum-exp per query
-  float red_m[2][4], red_l[2][4];
+  alignas(8) float lse_s[kNQ];  // pass 2: minus the log2-domain log-sum-exp per query (-inf for padding queries)
   float colsum_s[16][128];  // pass 1: per row-group column sums at the end of the slice
 };
 
@@ -100,7 +100,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   }
   if (PASS == 2 && tid < kNQ) {
     // log-sum-exp of query `tid` over the whole head: pass 1's per-slice (max, sum) pairs, merged in slice order
-    float lse = 0.f;
+    float lse = INFINITY;  // padding queries: exp2(anything - inf) = 0
     if (tid < g.L_q) {
       float m = -INFINITY, l = 0.f;
       for (int s = 0; s < g.n_slices; ++s) {
@@ -111,7 +111,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       }
       lse = m + log2f(l);
     }
-    sh->lse_s[tid] = lse;
+    sh->lse_s[tid] = -lse;
   }
   if (warp == 0) {
     tmem_alloc(smem_u32(&sh->tmem_base), 2 * kCols);
@@ -160,9 +160,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
       }
     }
-  } else if (warp < 4) {
+  } else if (warp < 4 || (PASS == 2 && warp < 8)) {
     // ---------------------------------------------------------------- logits out of tensor memory
-    const uint32_t t_lane = tmem + ((uint32_t)(warp * 32) << 16);
+    // (pass 2 has no key-vector work, so warps 4-7 are a second logit warpgroup: the two take alternate tiles,
+    // each the tensor-memory buffer of its own parity)
+    const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     if (PASS == 1) {
       const int q = tid;  // query row
       const bool row_ok = q < g.L_q;
@@ -214,7 +216,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     } else {
       // The mean key joins the queries as rows kNQ-2 (bf16 high part) and kNQ-1 (low part) of the Q tile, which
       // the copy zero-filled: generic-proxy writes, made visible to the tensor cores by the proxy fence.
-      mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
+      const int wg = warp >> 2, row = tid & 127;
+      if (wg == 0) mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
       if (tid < D) {
         float mk = 0.f;  // mean normalised key: pass 1's per-slice column sums, added in slice order
         for (int s = 0; s < g.n_slices; ++s) mk += g.colsum_part[((int64_t)hk * g.n_slices + s) * D + tid];
@@ -227,12 +230,15 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           *reinterpret_cast<__nv_bfloat16*>(q_tile + x * kAtomBytes + r * 128 + ((cc ^ (r & 7)) << 4) + e * 2) = part ? lo : hi;
         }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      mbar_arrive(smem_u32(&sh->q_patched));
+      if (wg == 0) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(smem_u32(&sh->q_patched));
+      }
       const float inv_nq = 1.f / (float)g.L_q, inv_lk = 1.f / (float)g.L_k;
-      for (int i = 0; i < n; ++i) {
+      const uint64_t sc2 = pack2(g.scale_log2, g.scale_log2);
+      for (int i = wg; i < n; i += 2) {
         const int b = i & 1;
-        const int tile_id = tile_of(i), j = tile_id * kKeys + tid;  // this thread's key
+        const int tile_id = tile_of(i), j = tile_id * kKeys + row;  // this thread's key
         const bool valid = j < g.L_k;
         const int64_t o = (int64_t)hk * g.L_k + j;
         const float n2 = valid && g.accum_phase != 1 ? g.norm2[o] : 0.f;  // in flight while the logits arrive
@@ -243,11 +249,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
-        float ms[4] = {0.f, 0.f, 0.f, 0.f};
+        // exp2(s * scale - lse) two queries at a time; lse_s holds -lse, and -inf for the padding queries (-> 0)
+        uint64_t ms2[2] = {0ull, 0ull};
 #pragma unroll
-        for (int q = 0; q < kNQ - 2; ++q)
-          if (q < g.L_q) ms[q & 3] += ex2(fmaf(__uint_as_float(sv[q]), g.scale_log2, -sh->lse_s[q]));
-        const float mass = ((ms[0] + ms[1]) + (ms[2] + ms[3])) * inv_nq;
+        for (int q = 0; q < kNQ - 2; q += 2) {
+          const uint64_t nl = *reinterpret_cast<const uint64_t*>(&sh->lse_s[q]);
+          float x0, x1;
+          unpack2(fma2(pack2(__uint_as_float(sv[q]), __uint_as_float(sv[q + 1])), sc2, nl), x0, x1);
+          ms2[(q >> 1) & 1] = add2(ms2[(q >> 1) & 1], pack2(ex2(x0), ex2(x1)));
+        }
+        float m0, m1, m2, m3;
+        unpack2(ms2[0], m0, m1);
+        unpack2(ms2[1], m2, m3);
+        const float mass = ((m0 + m1) + (m2 + m3)) * inv_nq;
         if (valid) {
           if (g.accum_phase == 1) {
             g.imp_accum[o] += mass;
@@ -267,29 +281,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
           a = dot * inv - (n2 * inv * inv) * inv_lk;
           g.a_out[o] = a;
         }
-        // softmax statistics (max, sum of exp) of a over the tile, fixed order
+        // softmax statistics (max, sum of exp) of a over this warp's 32 keys, fixed order
         float m = a;
 #pragma unroll
         for (int w = 16; w > 0; w >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, w));
         float l = valid ? expf(a - m) : 0.f;
 #pragma unroll
         for (int w = 16; w > 0; w >>= 1) l += __shfl_xor_sync(0xffffffffu, l, w);
-        if (lane == 0) {
-          sh->red_m[i & 1][warp] = m;
-          sh->red_l[i & 1][warp] = l;
-        }
-        named_barrier_128();
-        if (tid == 0) {
-          m = sh->red_m[i & 1][0];
-          l = sh->red_l[i & 1][0];
-          for (int w = 1; w < 4; ++w) {
-            const float m2 = sh->red_m[i & 1][w], l2 = sh->red_l[i & 1][w];
-            const float mn = fmaxf(m, m2);
-            l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (m2 == -INFINITY ? 0.f : l2 * expf(m2 - mn));
-            m = mn;
-          }
-          g.a_partial[hk * g.n_tiles + tile_id] = make_float2(m, l);
-        }
+        if (lane == 0) g.a_partial[((int64_t)hk * g.n_tiles + tile_id) * 4 + (warp & 3)] = make_float2(m, l);
       }
     }
   } else if (PASS == 1) {

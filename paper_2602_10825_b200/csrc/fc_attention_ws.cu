@@ -17,9 +17,10 @@
 // what lets the softmax warps rescale O_X in place when a row maximum moves.
 // The rescale is lazy: a row keeps its reference maximum until the true maximum exceeds it by more
 // than 2^8, so P stays below 256 and O is rescaled only a few times per row.
-// The softmax is written for issue slots and for the special-function unit, which at d = 128 is as
-// busy as the tensor pipe: three-input max, two-wide fp32 fma / add, one bf16x2 convert per
-// pair, and a share of the exponentials evaluated as a cubic on the fma pipe instead of ex2.
+// The softmax is written for issue slots: three-input max, two-wide fp32 fma / add, one bf16x2
+// convert per pair; every exponential is an ex2 (a cubic on the fma pipe for a share of them, and ex2 on
+// packed halves, were both measured slower: one warp per scheduler is bound by the latency of its own
+// instruction stream, and extra arithmetic lengthens it).
 // Every mbarrier wait is bounded (see mbar_wait_bounded); tensor memory is always released.
 #include <cmath>
 
@@ -36,11 +37,6 @@ constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {copy warp
 constexpr int kStages = 2;  // the MMA issuer computes stage and phase with masks: keep at 2
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
-// of every 32 columns, this many (the last ones) take the polynomial exponential
-#ifndef FC_ATTN_EMU_COLS
-#define FC_ATTN_EMU_COLS 0
-#endif
-constexpr int kEmuCols = FC_ATTN_EMU_COLS;
 // Registers per thread after the split: softmax warpgroups / the warpgroup of the copy and MMA warps.
 // The CTA owns 384 x 168 registers from launch (168 = what the launch bounds allow); setmaxnreg only moves
 // registers inside that pool, and an increase that the pool cannot cover would wait forever.
@@ -50,10 +46,6 @@ constexpr int kEmuCols = FC_ATTN_EMU_COLS;
 #endif
 static_assert(256 * FC_ATTN_REGS_HI + 128 * FC_ATTN_REGS_LO <= 384 * 168, "register split exceeds the CTA's pool");
 static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg takes multiples of 8");
-// how whole warps (softmax, copy) wait on a barrier: 0 every lane polls, 1 lane 0 polls, 2 lane 0 with a short sleep
-#ifndef FC_ATTN_WARP_WAIT
-#define FC_ATTN_WARP_WAIT 0
-#endif
 #ifndef FC_ATTN_STAGGER
 #define FC_ATTN_STAGGER 1
 #endif
@@ -68,13 +60,6 @@ constexpr int kPaceDelay = FC_ATTN_PACE_DELAY;
 #define FC_ATTN_SPECULATE 1
 #endif
 constexpr bool kSpeculate = FC_ATTN_SPECULATE != 0;
-// Option: two exponentials per special-function instruction (argument rounded to half precision, ex2 on the
-// packed pair).  Accuracy is unchanged (P is rounded to bf16 anyway), but the two extra conversions per pair cost
-// more issue slots than the special-function unit gains: measured slower on B200, so off.
-#ifndef FC_ATTN_EXP_F16X2
-#define FC_ATTN_EXP_F16X2 0
-#endif
-constexpr bool kExpF16x2 = FC_ATTN_EXP_F16X2 != 0;
 #define FC_STR2(x) #x
 #define FC_STR(x) FC_STR2(x)
 
@@ -98,47 +83,10 @@ struct Item {
   bool b_valid;  // tile B has at least one row of the chunk (false for the ragged last item of a chunk)
 };
 
-// 2^x for a pair through the packed half-precision ex2: x0 in the low half.  Arguments below -65504 are clamped
-// by the conversion's saturation to -inf -> 0.
-__device__ __forceinline__ void ex2_f16x2(float x0, float x1, float& y0, float& y1) {
-  uint32_t h;
-  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h) : "f"(x1), "f"(x0));
-  asm("ex2.approx.f16x2 %0, %0;" : "+r"(h));
-  asm("{\n.reg .b16 lo, hi;\nmov.b32 {lo, hi}, %2;\ncvt.f32.f16 %0, lo;\ncvt.f32.f16 %1, hi;\n}\n" : "=f"(y0), "=f"(y1) : "r"(h));
-}
-
-// 2^x for a pair, x <= 8, on the fma pipe: n = round(x) through the 1.5 * 2^23 shift, 2^(x-n) as a cubic
-// on [-0.5, 0.5] (relative error 7.5e-5, far below the bf16 rounding of P), then n added to the exponent
-// field.  Inputs below -126 are clamped; their result is a harmless ~1e-38.
-__device__ __forceinline__ void ex2_poly2(float x0, float x1, float& y0, float& y1) {
-  const uint64_t kShift = pack2(12582912.f, 12582912.f), kUnshift = pack2(-12582912.f, -12582912.f);
-  const uint64_t kMinus1 = pack2(-1.f, -1.f);
-  const uint64_t c0 = pack2(0.9999280572f, 0.9999280572f), c1 = pack2(0.6932609677f, 0.6932609677f);
-  const uint64_t c2 = pack2(0.2426111251f, 0.2426111251f), c3 = pack2(0.0551716685f, 0.0551716685f);
-  const uint64_t x = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-  const uint64_t t = add2(x, kShift);
-  const uint64_t n = add2(t, kUnshift);
-  const uint64_t f = fma2(n, kMinus1, x);
-  uint64_t p = fma2(c3, f, c2);
-  p = fma2(p, f, c1);
-  p = fma2(p, f, c0);
-  float p0, p1, t0, t1;
-  unpack2(p, p0, p1);
-  unpack2(t, t0, t1);
-  y0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
-  y1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
-}
-
 // P = 2^(S * scale - m) for one row of a 128-column tile, written back over S as bf16; returns the row sum.
-// With kWithMax the raw row maximum of the tile is computed on the side (into `raw_max`): the caller used the
-// reference it already had and checks afterwards whether the tile's maximum allows that.
-template <bool kAllEx2, bool kWithMax>
-__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s,
-                                          float& raw_max) {
+__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s) {
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t sum2[2] = {0ull, 0ull};
-  float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-  constexpr int kEmuPairs = kAllEx2 ? 0 : kEmuCols / 2;
 #pragma unroll
   for (int q2 = 0; q2 < kBN / 32; ++q2) {
     uint32_t pk[16];
@@ -146,38 +94,24 @@ __device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale
     for (int i = 0; i < 16; ++i) {
       const uint64_t x = fma2(pack2(__uint_as_float(sv[q2 * 32 + 2 * i]), __uint_as_float(sv[q2 * 32 + 2 * i + 1])),
                               sc2, nm2);
-      float x0, x1, p0, p1;
+      float x0, x1;
       unpack2(x, x0, x1);
-      if (kWithMax)
-        mx[i & 3] = max3(mx[i & 3], __uint_as_float(sv[q2 * 32 + 2 * i]), __uint_as_float(sv[q2 * 32 + 2 * i + 1]));
-      if (i >= 16 - kEmuPairs) {
-        ex2_poly2(x0, x1, p0, p1);
-      } else if (kExpF16x2 && !kAllEx2) {
-        ex2_f16x2(x0, x1, p0, p1);
-      } else {
-        p0 = ex2(x0);
-        p1 = ex2(x1);
-      }
+      const float p0 = ex2(x0), p1 = ex2(x1);
       sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
       pk[i] = cvt_bf16x2(p0, p1);
     }
     tmem_st16(t_s + q2 * 16, pk);
   }
-  if (kWithMax) raw_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
   float a, b, c, d;
   unpack2(sum2[0], a, b);
   unpack2(sum2[1], c, d);
   return (a + b) + (c + d);
 }
 
+// A wait by every lane of a warp (softmax and copy warps).  Measured alternatives: lane 0 polling with the
+// others parked at a warp barrier, and polls separated by nanosleep; both were slower or no faster.
 __device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort) {
-#if FC_ATTN_WARP_WAIT == 0
   mbar_wait_bounded(bar, parity, abort);
-#elif FC_ATTN_WARP_WAIT == 1
-  mbar_wait_warp(bar, parity, abort, 0);
-#else
-  mbar_wait_warp(bar, parity, abort, 32);
-#endif
 }
 
 template <int D>
@@ -488,13 +422,13 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
               tmem_st32(t_o + q4 * 32, r);
             }
           };
-          float alpha = 1.f, row_sum, raw_max = 0.f;
+          float alpha = 1.f, row_sum;
           if (kSpeculate && j > 0 && cols_valid == kBN) {
             // Common case: the reference maximum of the row does not move (it moves only when a tile exceeds it by
             // 2^8).  So exponentiate against the reference at once, without looking for the tile's maximum first.
             // A row whose tile sum stays below 2^8 cannot hold a term above 2^8; only if some row of the warp
             // exceeds that is the maximum computed, and the tile redone for the rows that have to move.
-            row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, raw_max);
+            row_sum = exp_tile(sv, scale_log2, m, t_s);
             if (__any_sync(0xffffffffu, !(row_sum <= 256.f))) {  // 2^kRescaleThreshold; also catches inf / NaN
               float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -511,7 +445,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                   m = tile_max;
                 }
                 rescale_o(alpha);
-                row_sum = exp_tile<false, false>(sv, scale_log2, m, t_s, raw_max);
+                row_sum = exp_tile(sv, scale_log2, m, t_s);
               }
             }
           } else {
@@ -535,9 +469,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
               m = tile_max;
             }
             if (j > 0 && __any_sync(0xffffffffu, move)) rescale_o(alpha);
-            // a ragged tile takes ex2 everywhere so that its masked columns give exactly 0
-            row_sum = cols_valid < kBN ? exp_tile<true, false>(sv, scale_log2, m, t_s, raw_max)
-                                       : exp_tile<false, false>(sv, scale_log2, m, t_s, raw_max);
+            row_sum = exp_tile(sv, scale_log2, m, t_s);  // masked columns: ex2(-inf) = 0 exactly
           }
           l = l * alpha + row_sum;
           tmem_wait_st();

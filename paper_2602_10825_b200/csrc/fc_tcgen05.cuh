@@ -63,27 +63,6 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
   return false;
 }
 
-// The same wait for a whole warp: lane 0 polls and the other lanes park at the warp barrier, so a waiting
-// warp costs one thread's worth of polling.  `backoff_ns` > 0 sleeps between polls.
-__device__ __forceinline__ void mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort,
-                                               uint32_t backoff_ns = 0) {
-  if ((threadIdx.x & 31) == 0) {
-    if (!mbar_try_wait(bar, parity)) {
-      const uint64_t t0 = global_timer_ns();
-      for (uint32_t n = 1;; ++n) {
-        if (backoff_ns) __nanosleep(backoff_ns);
-        if (mbar_try_wait(bar, parity)) break;
-        if (*abort) break;
-        if ((n & 31u) == 0 && global_timer_ns() - t0 > 2000000000ull) {
-          *abort = 1;
-          break;
-        }
-      }
-    }
-  }
-  __syncwarp();
-}
-
 // ---- TMA ------------------------------------------------------------------------------------
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
                                             int c2) {

@@ -9,18 +9,25 @@
 //   warp  8    scheduler + TMA       takes the next item off the counter, publishes it to the
 //                                    other warps through a 2-slot ring, then loads the Q pair and
 //                                    streams K and V tiles into 2-stage rings
-//   warps 9,10 MMA issuers           one thread per query tile: S_x(j), PV_x(j), S_x(j+1), ...; the tensor
-//                                    pipe runs the other tile's instructions while one tile is in softmax
-// Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512); P (bf16) overwrites the
-// low half of its S.  tcgen05.mma executes in issue order, so S_X(j+1) cannot overtake PV_X(j),
-// which still reads P_X(j), and "S_X(j) is complete" implies "PV_X(j-1) is complete", which is
-// what lets the softmax warps rescale O_X in place when a row maximum moves.
+//   warps 9,10 MMA issuers           one thread per query tile
+// Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
+// A key tile of 128 tokens is worked through as two halves of 64: S_x is two 64-column accumulators, each with
+// its own "full" and "P ready" barriers, and P (bf16) of a half overwrites the first 32 columns of that half.
+// The order of one MMA thread is S0(0) S1(0) | PV0(0) S0(1) PV1(0) S1(1) | PV0(1) S0(2) ..., so the S of the
+// next key tile's first half is issued as soon as P of this tile's first half has been handed to the tensor pipe,
+// while the softmax is still busy with the second half.  A softmax warp therefore finds its next half already
+// computed and never waits for a round trip through the tensor pipe: what bounds it is the special-function
+// unit (2 tiles x 128 x 128 exponentials at 16 per clock = 2048 clocks per pair of tiles, the same as the
+// tensor pipe's 2048).  With whole-tile S accumulators the chain S -> softmax -> PV -> S of one tile was the
+// critical path (about 3800 clocks per pair of tiles, measured).  The price: an S instruction with N = 64 reads
+// the whole 128-row Q operand from shared memory for half the columns and takes about 45 clocks instead of 32
+// (measured), so the tensor pipe needs about 1240 clocks per tile instead of 1024.
+// tcgen05.mma executes in issue order, so S_u(j+1) cannot overtake PV_u(j), which still reads P_u(j).
 // The rescale is lazy: a row keeps its reference maximum until the true maximum exceeds it by more
-// than 2^8, so P stays below 256 and O is rescaled only a few times per row.
+// than 2^8, so P stays below 256 and O is rescaled only a few times per row; a softmax warp that has to rescale
+// O_x first waits for the PV instructions issued so far (barrier pv_done: one phase per half).
 // The softmax is written for issue slots: three-input max, two-wide fp32 fma / add, one bf16x2
-// convert per pair; every exponential is an ex2 (a cubic on the fma pipe for a share of them, and ex2 on
-// packed halves, were both measured slower: one warp per scheduler is bound by the latency of its own
-// instruction stream, and extra arithmetic lengthens it).
+// convert per pair; every exponential is an ex2.
 // Every mbarrier wait is bounded (see mbar_wait_bounded); tensor memory is always released.
 #include <cmath>
 
@@ -33,6 +40,7 @@ namespace {
 using namespace fc::sm100;
 
 constexpr int kBM = 128, kBN = 128;
+constexpr int kHalf = kBN / 2;  // key columns per S accumulator
 constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {copy warp, two MMA warps, a spare warp}
 constexpr int kStages = 2;  // the MMA issuer computes stage and phase with masks: keep at 2
 constexpr uint32_t kTmemCols = 512;
@@ -46,15 +54,6 @@ constexpr float kRescaleThreshold = 8.f;  // log2 units
 #endif
 static_assert(256 * FC_ATTN_REGS_HI + 128 * FC_ATTN_REGS_LO <= 384 * 168, "register split exceeds the CTA's pool");
 static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg takes multiples of 8");
-#ifndef FC_ATTN_STAGGER
-#define FC_ATTN_STAGGER 1
-#endif
-constexpr bool kStagger = FC_ATTN_STAGGER != 0;
-// clocks between the S groups of the two query tiles (see the pacing comment in the MMA threads)
-#ifndef FC_ATTN_PACE_DELAY
-#define FC_ATTN_PACE_DELAY 1100
-#endif
-constexpr int kPaceDelay = FC_ATTN_PACE_DELAY;
 // exponentiate against the running reference before the tile's maximum is known (see the softmax loop)
 #ifndef FC_ATTN_SPECULATE
 #define FC_ATTN_SPECULATE 1
@@ -66,11 +65,11 @@ constexpr bool kSpeculate = FC_ATTN_SPECULATE != 0;
 struct WsSmem {
   uint64_t q_full, q_empty;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], p_ready[2], o_done[2];
+  uint64_t s_full[2][2], p_ready[2][2];  // [query tile][half of the key tile]
+  uint64_t pv_done[2];                   // per query tile: one phase per PV half, in issue order
+  uint64_t o_done[2];                    // per query tile: one phase per item, after its last PV
   uint64_t it_full[2], it_empty[2];
   int32_t it_slot[2];
-  uint32_t s_issued[2];   // per query tile: number of S groups its MMA thread has issued (pacing hint) ...
-  uint32_t s_clock[2];    // ... and the SM clock at the last of them
   uint32_t tmem_base;
   uint32_t abort;
   int32_t n_act, total_items;
@@ -83,12 +82,13 @@ struct Item {
   bool b_valid;  // tile B has at least one row of the chunk (false for the ragged last item of a chunk)
 };
 
-// P = 2^(S * scale - m) for one row of a 128-column tile, written back over S as bf16; returns the row sum.
-__device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale_log2, float m, uint32_t t_s) {
+// P = 2^(S * scale - m) for one row of a 64-column half tile, written as bf16 to tensor-memory columns
+// [t_p, t_p + 32); returns the row sum.
+__device__ __forceinline__ float exp_half(const uint32_t (&sv)[kHalf], float scale_log2, float m, uint32_t t_p) {
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
-  for (int q2 = 0; q2 < kBN / 32; ++q2) {
+  for (int q2 = 0; q2 < kHalf / 32; ++q2) {
     uint32_t pk[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
@@ -100,7 +100,7 @@ __device__ __forceinline__ float exp_tile(const uint32_t (&sv)[kBN], float scale
       sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
       pk[i] = cvt_bf16x2(p0, p1);
     }
-    tmem_st16(t_s + q2 * 16, pk);
+    tmem_st16(t_p + q2 * 16, pk);
   }
   float a, b, c, d;
   unpack2(sum2[0], a, b);
@@ -141,8 +141,11 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       mbar_init(smem_u32(&sh->v_empty[s]), 2);
     }
     for (int x = 0; x < 2; ++x) {
-      mbar_init(smem_u32(&sh->s_full[x]), 1);
-      mbar_init(smem_u32(&sh->p_ready[x]), 4);  // one arrival per softmax warp
+      for (int u = 0; u < 2; ++u) {
+        mbar_init(smem_u32(&sh->s_full[x][u]), 1);
+        mbar_init(smem_u32(&sh->p_ready[x][u]), 4);  // one arrival per softmax warp
+      }
+      mbar_init(smem_u32(&sh->pv_done[x]), 1);
       mbar_init(smem_u32(&sh->o_done[x]), 1);
       mbar_init(smem_u32(&sh->it_full[x]), 1);
       mbar_init(smem_u32(&sh->it_empty[x]), 10);  // the two MMA threads and the eight softmax warps
@@ -150,8 +153,6 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     }
     mbar_fence_init();
     sh->abort = 0;
-    sh->s_issued[0] = sh->s_issued[1] = 0;
-    sh->s_clock[0] = sh->s_clock[1] = 0;
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
     tma_prefetch_desc(&tmap_v);
@@ -282,60 +283,35 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   } else if (warp == 9 || warp == 10) {
     // ------------------------------------------------------------------ MMA issuers (one thread per query tile)
     // Lane 0 of warp 9 issues S_A and PV_A, lane 0 of warp 10 issues S_B and PV_B.  The tensor pipe takes
-    // instructions in arrival order; the order that matters, S_x(j+1) after PV_x(j), is program order of one
-    // thread.  While one thread sits in a wait or a commit the other keeps the pipe fed, and neither is held up
-    // by the other tile's softmax.
+    // instructions in arrival order; the order that matters, S_u(j+1) after PV_u(j), is program order of one
+    // thread.  While one thread sits in a wait or a commit the other keeps the pipe fed.
     if (lane == 0) {
     const int x = warp - 9;
-    constexpr uint32_t kIdescQK = idesc_bf16_f32(kBM, kBN, false, false);
+    constexpr uint32_t kIdescQK = idesc_bf16_f32(kBM, kHalf, false, false);
     constexpr uint32_t kIdescPV = idesc_bf16_f32(kBM, D, false, true);
     // descriptors are built once; a k-step only moves the 14-bit address field (units of 16 bytes)
     const uint64_t dq = smem_desc_sw128(q_s + x * kTileBytes, 16, 1024), dk = smem_desc_sw128(k_s, 16, 1024),
                    dv = smem_desc_sw128(v_s, kAtomBytes, 1024);
     const uint32_t t_s = tmem + x * 128, t_o = tmem + 256 + x * 128;
-    auto issue_s = [&](uint32_t st) {  // S_x = Q_x K^T
-      const uint64_t b0 = dk + (uint64_t)(st * (kTileBytes >> 4));
+    auto issue_s = [&](uint32_t st, int u) {  // S_x[:, half u] = Q_x K[half u]^T; a key row is 128 bytes of each atom
+      const uint64_t b0 = dk + (uint64_t)((st * kTileBytes + u * (kHalf * 128)) >> 4);
 #pragma unroll
       for (int kk = 0; kk < D / 16; ++kk) {
         const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
-        umma_ss(t_s, dq + off, b0 + off, kIdescQK, kk > 0);
+        umma_ss(t_s + u * kHalf, dq + off, b0 + off, kIdescQK, kk > 0);
       }
     };
-    auto issue_pv = [&](uint32_t st, bool accumulate) {  // O_x (+)= P_x V
-      const uint64_t b0 = dv + (uint64_t)(st * (kTileBytes >> 4));
+    auto issue_pv = [&](uint32_t st, int u, bool accumulate) {  // O_x (+)= P_x[:, half u] V[half u]
+      const uint64_t b0 = dv + (uint64_t)((st * kTileBytes + u * (kHalf / 16) * 2048) >> 4);
 #pragma unroll
-      for (int kk = 0; kk < kBN / 16; ++kk)
-        umma_ts(t_o, t_s + kk * 8, b0 + (uint64_t)(kk * (2048 >> 4)), kIdescPV, accumulate || kk > 0);
+      for (int kk = 0; kk < kHalf / 16; ++kk)
+        umma_ts(t_o, t_s + u * kHalf + kk * 8, b0 + (uint64_t)(kk * (2048 >> 4)), kIdescPV, accumulate || kk > 0);
     };
     // barrier addresses as plain registers: the issue loop should be little more than the MMAs themselves
     const uint32_t b_kfull = smem_u32(&sh->k_full[0]), b_kempty = smem_u32(&sh->k_empty[0]);
     const uint32_t b_vfull = smem_u32(&sh->v_full[0]), b_vempty = smem_u32(&sh->v_empty[0]);
-    const uint32_t b_sfull = smem_u32(&sh->s_full[x]), b_pready = smem_u32(&sh->p_ready[x]);
-    // Pacing.  Left alone, the two tiles fall into step: both softmaxes run together, sharing the special-
-    // function unit, and then both tiles' MMAs queue up behind each other.  So each S is issued no earlier than
-    // kPaceDelay clocks after the other tile's S for its current key tile was issued: S_B(j) after S_A(j),
-    // S_A(j+1) after S_B(j).  That keeps the two softmaxes apart by a good part of a period, and one tile's MMAs
-    // run under the other tile's softmax.  The MMA threads time each other directly (their instruction streams
-    // are short and ordered); it is only a delay: no data depends on it, and it gives up after 20 us.
-    auto pace = [&](uint32_t want) {
-      if (!kStagger) return;
-      volatile uint32_t* issued = &sh->s_issued[x ^ 1];
-      volatile uint32_t* clk = &sh->s_clock[x ^ 1];
-      if ((int32_t)(*issued - want) < 0) {  // the global timer is slow to read: only when there is something to wait for
-        const uint64_t t0 = global_timer_ns();
-        while ((int32_t)(*issued - want) < 0) {
-          if (global_timer_ns() - t0 > 20000ull) return;
-        }
-      }
-      if (*issued != want) return;  // the other tile is further ahead than that: no need to wait
-      const uint32_t since = *clk;
-      while ((uint32_t)clock64() - since < (uint32_t)kPaceDelay) {
-      }
-    };
-    auto announce = [&](uint32_t n_issued, uint32_t back_date) {
-      *(volatile uint32_t*)&sh->s_clock[x] = (uint32_t)clock64() - back_date;
-      *(volatile uint32_t*)&sh->s_issued[x] = n_issued;
-    };
+    const uint32_t b_sfull = smem_u32(&sh->s_full[x][0]), b_pready = smem_u32(&sh->p_ready[x][0]);
+    const uint32_t b_pvdone = smem_u32(&sh->pv_done[x]);
     // Barrier phases are counted per use: tile B sits out the items in which it has no rows (the last item of a
     // chunk whose length is not a multiple of 256), so its barriers see fewer phases than tile A's.
     uint32_t kv = 0, uses = 0;
@@ -351,32 +327,52 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       tc_fence_after();
       if (x == 1 && !it.b_valid) {
         // Nothing to compute for tile B.  Its arrivals on the ring barriers are still due, one stage at a time
-        // (waiting for the stage to be full keeps them in the right phase), and tile A still paces itself on it.
+        // (waiting for the stage to be full keeps them in the right phase).
         for (int j = 0; j < n_tiles; ++j, ++kv) {
           const uint32_t st = kv & 1, ph = (kv >> 1) & 1;
           mbar_wait_bounded(b_kfull + 8 * st, ph, abort);
           mbar_arrive(b_kempty + 8 * st);
           mbar_wait_bounded(b_vfull + 8 * st, ph, abort);
           mbar_arrive(b_vempty + 8 * st);
-          if (kStagger) announce(kv + 1, kPaceDelay);
         }
         mbar_arrive(smem_u32(&sh->q_empty));
         continue;
       }
-      for (int j = 0; j < n_tiles; ++j, ++kv, ++uses) {
+      if (n_tiles > 0) {  // both halves of S for the first key tile
         const uint32_t st = kv & 1, ph = (kv >> 1) & 1;  // kStages == 2
         mbar_wait_bounded(b_kfull + 8 * st, ph, abort);
-        pace(kv + x);
         tc_fence_after();
-        issue_s(st);
+        issue_s(st, 0);
         umma_commit(b_sfull);
+        issue_s(st, 1);
+        umma_commit(b_sfull + 8);
         umma_commit(b_kempty + 8 * st);
-        if (kStagger) announce(kv + 1, 0);
+      }
+      for (int j = 0; j < n_tiles; ++j, ++kv, ++uses) {
+        const uint32_t st = kv & 1, ph = (kv >> 1) & 1;
+        const uint32_t st2 = st ^ 1, ph2 = ((kv + 1) >> 1) & 1;  // the next key tile's stage
+        const bool more = j + 1 < n_tiles;
         mbar_wait_bounded(b_vfull + 8 * st, ph, abort);
         mbar_wait_bounded(b_pready, uses & 1, abort);
         tc_fence_after();
-        issue_pv(st, j > 0);
+        issue_pv(st, 0, j > 0);
+        umma_commit(b_pvdone);
+        if (more) {
+          mbar_wait_bounded(b_kfull + 8 * st2, ph2, abort);
+          tc_fence_after();
+          issue_s(st2, 0);
+          umma_commit(b_sfull);
+        }
+        mbar_wait_bounded(b_pready + 8, uses & 1, abort);
+        tc_fence_after();
+        issue_pv(st, 1, true);
+        umma_commit(b_pvdone);
         umma_commit(b_vempty + 8 * st);
+        if (more) {
+          issue_s(st2, 1);
+          umma_commit(b_sfull + 8);
+          umma_commit(b_kempty + 8 * st2);
+        }
       }
       umma_commit(smem_u32(&sh->q_empty));  // every read of this thread's Q tile has been issued
       umma_commit(smem_u32(&sh->o_done[x]));
@@ -392,7 +388,25 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const uint32_t t_o = tmem + lane_base + 256 + x * 128;
     const int r_in = (warp & 3) * 32 + lane;  // row inside the tile
     const float scale_log2 = g.scale * 1.4426950408889634f;
-    uint32_t kv = 0, uses = 0, items = 0;  // tiles seen, tiles and items actually processed (barrier phases)
+    // tiles seen; tiles, half tiles and items actually processed (barrier phases)
+    uint32_t kv = 0, uses = 0, sub = 0, items = 0;
+    // Before O_x is rescaled in place: every PV instruction that this warp has released so far (the first `sub`
+    // phases of pv_done) has completed.  A parity wait tells two states apart, and there are only two here: the
+    // half tile being worked on was computed after PV of two halves ago, so at least sub - 1 phases are over.
+    auto wait_pv = [&]() {
+      warp_wait(smem_u32(&sh->pv_done[x]), (sub - 1) & 1, abort);
+      tc_fence_after();
+    };
+    auto rescale_o = [&](float alpha) {
+#pragma unroll
+      for (int q4 = 0; q4 < D / 32; ++q4) {
+        uint32_t r[32];
+        tmem_ld32_wait(t_o + q4 * 32, r);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+        tmem_st32(t_o + q4 * 32, r);
+      }
+    };
     for (uint32_t it_n = 0;; ++it_n) {
       const int item = next_item(it_n);
       if (item < 0) break;
@@ -408,74 +422,71 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         if (seg_vis <= 0) break;
         for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv, ++j, ++uses) {
           const int cols_valid = min(kBN, seg_vis - j0);
-          warp_wait(smem_u32(&sh->s_full[x]), uses & 1, abort);
-          tc_fence_after();
-          uint32_t sv[kBN];
-          tmem_ld128_wait(t_s, sv);
-          auto rescale_o = [&](float alpha) {
 #pragma unroll
-            for (int q4 = 0; q4 < D / 32; ++q4) {
-              uint32_t r[32];
-              tmem_ld32_wait(t_o + q4 * 32, r);
-#pragma unroll
-              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-              tmem_st32(t_o + q4 * 32, r);
-            }
-          };
-          float alpha = 1.f, row_sum;
-          if (kSpeculate && j > 0 && cols_valid == kBN) {
-            // Common case: the reference maximum of the row does not move (it moves only when a tile exceeds it by
-            // 2^8).  So exponentiate against the reference at once, without looking for the tile's maximum first.
-            // A row whose tile sum stays below 2^8 cannot hold a term above 2^8; only if some row of the warp
-            // exceeds that is the maximum computed, and the tile redone for the rows that have to move.
-            row_sum = exp_tile(sv, scale_log2, m, t_s);
-            if (__any_sync(0xffffffffu, !(row_sum <= 256.f))) {  // 2^kRescaleThreshold; also catches inf / NaN
+          for (int u = 0; u < 2; ++u, ++sub) {
+            const int mine_valid = min(max(cols_valid - u * kHalf, 0), kHalf);
+            const uint32_t t_su = t_s + u * kHalf;  // S of this half; its first 32 columns take P
+            const bool first = j == 0 && u == 0;
+            warp_wait(smem_u32(&sh->s_full[x][u]), uses & 1, abort);
+            tc_fence_after();
+            uint32_t sv[kHalf];
+            tmem_ld64_wait(t_su, sv);
+            auto row_max = [&]() {
               float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-              for (int i = 0; i < kBN; i += 8) {
+              for (int i = 0; i < kHalf; i += 8) {
 #pragma unroll
                 for (int c4 = 0; c4 < 4; ++c4)
                   mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
               }
-              const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
-              const bool move = tile_max > m + kRescaleThreshold;
-              if (__any_sync(0xffffffffu, move)) {
-                if (move) {
-                  alpha = ex2(m - tile_max);
-                  m = tile_max;
+              return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
+            };
+            float alpha = 1.f, row_sum;
+            if (kSpeculate && !first && mine_valid == kHalf) {
+              // Common case: the reference maximum of the row does not move (it moves only when a half tile exceeds
+              // it by 2^8).  So exponentiate against the reference at once, without looking for the maximum first.
+              // A row whose sum stays below 2^8 cannot hold a term above 2^8; only if some row of the warp
+              // exceeds that is the maximum computed, and the half tile redone for the rows that have to move.
+              row_sum = exp_half(sv, scale_log2, m, t_su);
+              if (__any_sync(0xffffffffu, !(row_sum <= 256.f))) {  // 2^kRescaleThreshold; also catches inf / NaN
+                const float tile_max = row_max();
+                const bool move = tile_max > m + kRescaleThreshold;
+                if (__any_sync(0xffffffffu, move)) {
+                  if (move) {
+                    alpha = ex2(m - tile_max);
+                    m = tile_max;
+                  }
+                  tmem_wait_st();
+                  wait_pv();
+                  rescale_o(alpha);
+                  row_sum = exp_half(sv, scale_log2, m, t_su);
                 }
-                rescale_o(alpha);
-                row_sum = exp_tile(sv, scale_log2, m, t_s);
               }
-            }
-          } else {
-            if (cols_valid < kBN) {
+            } else {
+              if (mine_valid < kHalf) {
 #pragma unroll
-              for (int i = 0; i < kBN; ++i)
-                if (i >= cols_valid) sv[i] = 0xff800000u;  // -inf
+                for (int i = 0; i < kHalf; ++i)
+                  if (i >= mine_valid) sv[i] = 0xff800000u;  // -inf
+              }
+              const float tile_max = row_max();  // -inf if the half holds no visible token: then nothing moves
+              // lazy reference update: move only when the maximum grew by more than the threshold
+              const bool move = tile_max > m + kRescaleThreshold;  // always true on an item's first half (m = -inf)
+              if (move) {
+                alpha = ex2(m - tile_max);
+                m = tile_max;
+              }
+              if (!first && __any_sync(0xffffffffu, move)) {
+                wait_pv();
+                rescale_o(alpha);
+              }
+              row_sum = exp_half(sv, scale_log2, m, t_su);  // masked columns: ex2(-inf) = 0 exactly
             }
-            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int i = 0; i < kBN; i += 8) {
-#pragma unroll
-              for (int c4 = 0; c4 < 4; ++c4)
-                mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
-            }
-            const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
-            // lazy reference update: move only when the maximum grew by more than the threshold
-            const bool move = tile_max > m + kRescaleThreshold;  // always true on the first tile (m = -inf)
-            if (move) {
-              alpha = ex2(m - tile_max);
-              m = tile_max;
-            }
-            if (j > 0 && __any_sync(0xffffffffu, move)) rescale_o(alpha);
-            row_sum = exp_tile(sv, scale_log2, m, t_s);  // masked columns: ex2(-inf) = 0 exactly
+            l = l * alpha + row_sum;
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready[x][u]));
           }
-          l = l * alpha + row_sum;
-          tmem_wait_st();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&sh->p_ready[x]));
         }
       }
       // epilogue

@@ -27,7 +27,12 @@
 // than 2^8, so P stays below 256 and O is rescaled only a few times per row; a softmax warp that has to rescale
 // O_x first waits for the PV instructions issued so far (barrier pv_done: one phase per half).
 // The softmax is written for issue slots: three-input max, two-wide fp32 fma / add, one bf16x2
-// convert per pair; every exponential is an ex2.
+// convert per pair.  Two softmax warps share a scheduler (the same lane quadrant of tiles A and B), and together
+// they saturate the special-function unit (measured: 1115 clocks per half tile per warp when both run, 640 when
+// one runs alone).  One column pair in four therefore takes its exponential on the fma pipe (range reduction and a
+// cubic): 900 clocks per half tile in isolation; a larger share costs more fma-pipe time than it saves.
+// As measured with clock probes, a softmax warp now spends about 75 % of its time in exponentials and 10 % waiting
+// for S; the tensor pipe has work about 75 % of the time.
 // Every mbarrier wait is bounded (see mbar_wait_bounded); tensor memory is always released.
 #include <cmath>
 
@@ -49,8 +54,8 @@ constexpr float kRescaleThreshold = 8.f;  // log2 units
 // The CTA owns 384 x 168 registers from launch (168 = what the launch bounds allow); setmaxnreg only moves
 // registers inside that pool, and an increase that the pool cannot cover would wait forever.
 #ifndef FC_ATTN_REGS_HI
-#define FC_ATTN_REGS_HI 216
-#define FC_ATTN_REGS_LO 72
+#define FC_ATTN_REGS_HI 200
+#define FC_ATTN_REGS_LO 104
 #endif
 static_assert(256 * FC_ATTN_REGS_HI + 128 * FC_ATTN_REGS_LO <= 384 * 168, "register split exceeds the CTA's pool");
 static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg takes multiples of 8");
@@ -137,6 +142,75 @@ __device__ __forceinline__ float exp_half(const uint32_t (&sv)[kHalf], float sca
   unpack2(sum2[0], a, b);
   unpack2(sum2[1], c, d);
   return (a + b) + (c + d);
+}
+
+// Groups of MMAs issued as one block of instructions, every operand already in a register.  The issuing thread
+// does not run ahead of the tensor pipe: what it executes between two MMAs of its own is time during which the
+// pipe has nothing from it (measured: 64 clocks per 128x128x16 MMA back to back, plus 6 to 9 clocks for every
+// instruction in between).  So descriptors are computed, and pinned in registers, before the wait that precedes a group.
+template <int N>
+__device__ __forceinline__ void pin(uint64_t (&d)[N]) {
+  static_assert(N == 4 || N == 8, "group size");
+  if constexpr (N == 8)
+    asm volatile("" : "+l"(d[0]), "+l"(d[1]), "+l"(d[2]), "+l"(d[3]), "+l"(d[4]), "+l"(d[5]), "+l"(d[6]), "+l"(d[7]));
+  else
+    asm volatile("" : "+l"(d[0]), "+l"(d[1]), "+l"(d[2]), "+l"(d[3]));
+}
+__device__ __forceinline__ void pin(uint32_t (&d)[4]) {
+  asm volatile("" : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]));
+}
+// D = A B over N k-steps, A and B in shared memory; the first k-step overwrites D
+template <int N>
+__device__ __forceinline__ void umma_ss_group(uint32_t d_tmem, const uint64_t (&a)[N], const uint64_t (&b)[N], uint32_t idesc) {
+  if constexpr (N == 8) {
+    asm volatile(
+        "{\n"
+        ".reg .pred f, t;\n"
+        "setp.ne.b32 f, %0, %0;\n"
+        "setp.eq.b32 t, %0, %0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %10, %1, f;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %11, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %12, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %5, %13, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %6, %14, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %7, %15, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %8, %16, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %9, %17, %1, t;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(idesc), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]),
+          "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7])
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n"
+        ".reg .pred f, t;\n"
+        "setp.ne.b32 f, %0, %0;\n"
+        "setp.eq.b32 t, %0, %0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %6, %1, f;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %7, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %8, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %5, %9, %1, t;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(idesc), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3])
+        : "memory");
+  }
+}
+// D (+)= A B over 4 k-steps, A in tensor memory; the first k-step accumulates only if `accumulate`
+__device__ __forceinline__ void umma_ts_group(uint32_t d_tmem, const uint32_t (&a)[4], const uint64_t (&b)[4], uint32_t idesc,
+                                              uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p, t;\n"
+      "setp.ne.b32 p, %2, 0;\n"
+      "setp.eq.b32 t, %0, %0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%3], %7, %1, p;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%4], %8, %1, t;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%5], %9, %1, t;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%6], %10, %1, t;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(idesc), "r"(accumulate), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]),
+        "l"(b[3])
+      : "memory");
 }
 
 // A wait by every lane of a warp (softmax and copy warps).  Measured alternatives: lane 0 polling with the
@@ -324,20 +398,32 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     const uint64_t dq = smem_desc_sw128(q_s + x * kTileBytes, 16, 1024), dk = smem_desc_sw128(k_s, 16, 1024),
                    dv = smem_desc_sw128(v_s, kAtomBytes, 1024);
     const uint32_t t_s = tmem + x * 128, t_o = tmem + 256 + x * 128;
-    auto issue_s = [&](uint32_t st, int u) {  // S_x[:, half u] = Q_x K[half u]^T; a key row is 128 bytes of each atom
+    constexpr int kSteps = D / 16;
+    uint64_t qa[kSteps], kb[kSteps], vb[4];  // operand descriptors of the next S group (Q_x fixed) and PV group
+    uint32_t pa[4];                          // tensor-memory addresses of P for the next PV group
+#pragma unroll
+    for (int kk = 0; kk < kSteps; ++kk) qa[kk] = dq + (uint64_t)(((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4);
+    pin(qa);
+    // S_x[:, half u] = Q_x K[half u]^T; a key row is 128 bytes of each atom
+    auto prep_s = [&](uint32_t st, int u) {
       const uint64_t b0 = dk + (uint64_t)((st * kTileBytes + u * (kHalf * 128)) >> 4);
 #pragma unroll
-      for (int kk = 0; kk < D / 16; ++kk) {
-        const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
-        umma_ss(t_s + u * kHalf, dq + off, b0 + off, kIdescQK, kk > 0);
-      }
+      for (int kk = 0; kk < kSteps; ++kk) kb[kk] = b0 + (uint64_t)(((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4);
+      pin(kb);
     };
-    auto issue_pv = [&](uint32_t st, int u, bool accumulate) {  // O_x (+)= P_x[:, half u] V[half u]
+    auto issue_s = [&](int u) { umma_ss_group<kSteps>(t_s + u * kHalf, qa, kb, kIdescQK); };
+    // O_x (+)= P_x[:, half u] V[half u]
+    auto prep_pv = [&](uint32_t st, int u) {
       const uint64_t b0 = dv + (uint64_t)((st * kTileBytes + u * (kHalf / 16) * 2048) >> 4);
 #pragma unroll
-      for (int kk = 0; kk < kHalf / 16; ++kk)
-        umma_ts(t_o, t_s + u * kHalf + kk * 8, b0 + (uint64_t)(kk * (2048 >> 4)), kIdescPV, accumulate || kk > 0);
+      for (int kk = 0; kk < 4; ++kk) {
+        vb[kk] = b0 + (uint64_t)(kk * (2048 >> 4));
+        pa[kk] = t_s + u * kHalf + kk * 8;
+      }
+      pin(vb);
+      pin(pa);
     };
+    auto issue_pv = [&](bool accumulate) { umma_ts_group(t_o, pa, vb, kIdescPV, accumulate); };
     // barrier addresses as plain registers: the issue loop should be little more than the MMAs themselves
     const uint32_t b_kfull = smem_u32(&sh->k_full[0]), b_kempty = smem_u32(&sh->k_empty[0]);
     const uint32_t b_vfull = smem_u32(&sh->v_full[0]), b_vempty = smem_u32(&sh->v_empty[0]);
@@ -371,11 +457,13 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       }
       if (n_tiles > 0) {  // both halves of S for the first key tile
         const uint32_t st = kv & 1, ph = (kv >> 1) & 1;  // kStages == 2
+        prep_s(st, 0);
         mbar_wait_bounded(b_kfull + 8 * st, ph, abort);
         tc_fence_after();
-        issue_s(st, 0);
+        issue_s(0);
         umma_commit(b_sfull);
-        issue_s(st, 1);
+        prep_s(st, 1);
+        issue_s(1);
         umma_commit(b_sfull + 8);
         umma_commit(b_kempty + 8 * st);
       }
@@ -383,24 +471,28 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         const uint32_t st = kv & 1, ph = (kv >> 1) & 1;
         const uint32_t st2 = st ^ 1, ph2 = ((kv + 1) >> 1) & 1;  // the next key tile's stage
         const bool more = j + 1 < n_tiles;
+        prep_pv(st, 0);
+        if (more) prep_s(st2, 0);
         mbar_wait_bounded(b_vfull + 8 * st, ph, abort);
         mbar_wait_bounded(b_pready, uses & 1, abort);
         tc_fence_after();
-        issue_pv(st, 0, j > 0);
+        issue_pv(j > 0);
         umma_commit(b_pvdone);
         if (more) {
           mbar_wait_bounded(b_kfull + 8 * st2, ph2, abort);
           tc_fence_after();
-          issue_s(st2, 0);
+          issue_s(0);
           umma_commit(b_sfull);
         }
+        prep_pv(st, 1);
+        if (more) prep_s(st2, 1);
         mbar_wait_bounded(b_pready + 8, uses & 1, abort);
         tc_fence_after();
-        issue_pv(st, 1, true);
+        issue_pv(true);
         umma_commit(b_pvdone);
         umma_commit(b_vempty + 8 * st);
         if (more) {
-          issue_s(st2, 1);
+          issue_s(1);
           umma_commit(b_sfull + 8);
           umma_commit(b_kempty + 8 * st2);
         }

@@ -4,7 +4,12 @@
 // Two pipelines, both deterministic (no floating-point atomics).  bf16 inputs with one query head per key head
 // and at most 62 observation queries take the tensor-core kernels of fc_score_tc.cu followed by the finalize
 // kernel below; everything else (fp32, grouped query heads, more queries) takes the
-// CUDA-core pipeline, deterministic (no floating-point atomics), five launches per call:
+// CUDA-core pipeline (below).  bf16 inputs with more than 128 observation queries per key head (a latent frame
+// or a whole chunk of them) take the frame-level pipeline: key norms and mean key by the CUDA-core pass-1 kernel
+// without queries, every query's log-sum-exp over the candidates by the chunk-attention kernel (its LSE output;
+// its O output goes to scratch), the attention mass by the tensor-core kernel of fc_score_frame.cu, then the
+// CUDA-core pass-2 kernel fed with that mass, and the finalize kernel.
+// The CUDA-core pipeline, five launches per call:
 //   pass1     one thread per key: raw logits of all observation queries against its key,
 //             written to the workspace; normalised key summed per 128-key tile (mean key)
 //   row_lse   one block per (head, query): log-sum-exp of that query's logits over all keys
@@ -15,12 +20,14 @@
 //   finalize  softmax of a over the head, max-pool of the importance, lambda-mix
 #include <cmath>
 
+#include "fc_attention.cuh"
 #include "fc_common.cuh"
 #include "fc_score.cuh"
 
 namespace {
 
 constexpr int kTile = 128;  // keys per block, one thread each
+constexpr int kCoreMaxQueries = 128;  // query rows per key head that the CUDA-core pipeline holds in shared memory
 
 template <typename T, int D>
 __device__ __forceinline__ void load_row(const T* __restrict__ row, float (&x)[D]) {
@@ -168,6 +175,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kTile)
 score_pass2_kernel(const T* __restrict__ K, ScoreGeom g, const float* __restrict__ S,
                    const float* __restrict__ lse, const float* __restrict__ mean_key,
+                   const float* __restrict__ mass_in,  // frame-level path: sum over the queries already taken
                    float* __restrict__ imp_accum, int accum_phase, int n_steps,
                    float* __restrict__ imp_out, float* __restrict__ a_out, float2* __restrict__ a_partial) {
   __shared__ float mk_s[D];
@@ -175,17 +183,21 @@ score_pass2_kernel(const T* __restrict__ K, ScoreGeom g, const float* __restrict
   __shared__ float sm_m[kTile / 32], sm_l[kTile / 32];
   const int hk = blockIdx.y, tile = blockIdx.x, tid = threadIdx.x;
   if (tid < D) mk_s[tid] = mean_key[hk * D + tid];
-  if (tid < g.n_q) lse_s[tid] = lse[hk * g.n_q + tid];
+  if (!mass_in && tid < g.n_q) lse_s[tid] = lse[hk * g.n_q + tid];
   __syncthreads();
   const int j = tile * kTile + tid;
   const bool valid = j < g.L_k;
   float a = -INFINITY;
   if (valid) {
-    const float* s = S + ((int64_t)hk * g.n_q) * g.L_k + j;
-    float mass = 0.f;
-    for (int i = 0; i < g.n_q; ++i) mass += expf(s[(int64_t)i * g.L_k] - lse_s[i]);
-    mass /= (float)g.n_q;
     const int64_t o = (int64_t)hk * g.L_k + j;
+    float mass = 0.f;
+    if (mass_in) {
+      mass = mass_in[o];
+    } else {
+      const float* s = S + ((int64_t)hk * g.n_q) * g.L_k + j;
+      for (int i = 0; i < g.n_q; ++i) mass += expf(s[(int64_t)i * g.L_k] - lse_s[i]);
+    }
+    mass /= (float)g.n_q;
     if (accum_phase == 1) {
       imp_accum[o] += mass;
     } else if (accum_phase == 2) {
@@ -261,6 +273,11 @@ struct ScoreWs {
   float* tc_colsum;   // per-slice sums of normalised keys
   float* tc_lse2;
   float* tc_norm2;
+  // frame-level path
+  void* fr_O;          // scratch output of the attention launch that produces the log-sum-exps
+  float* fr_mass;      // [H, L_k] sum over the queries of exp(logit - lse)
+  int32_t* fr_ctl;     // active_ids[1] = 0, n_active = 1
+  void* fr_attn_ws;
   size_t total;
 };
 
@@ -272,7 +289,8 @@ ScoreWs carve(const ScoreGeom& g, void* ws) {
     off += fc::align_up(bytes, 256);
     return p;
   };
-  w.S = (float*)take((size_t)g.H_kv * g.n_q * g.L_k * 4);
+  const bool frame = g.n_q > kCoreMaxQueries;
+  w.S = (float*)take(frame ? 0 : (size_t)g.H_kv * g.n_q * g.L_k * 4);
   w.mk_partial = (float*)take((size_t)g.H_kv * g.n_tiles * g.d * 4);
   w.lse = (float*)take((size_t)g.H_kv * g.n_q * 4);
   w.mean_key = (float*)take((size_t)g.H_kv * g.d * 4);
@@ -283,6 +301,10 @@ ScoreWs carve(const ScoreGeom& g, void* ws) {
   w.tc_colsum = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * g.d * 4);
   w.tc_lse2 = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxQueries * 4);
   w.tc_norm2 = (float*)take((size_t)g.H_kv * g.L_k * 4);
+  w.fr_O = take(frame ? (size_t)g.H_kv * g.L_q * g.d * 2 : 0);
+  w.fr_mass = (float*)take(frame ? (size_t)g.H_kv * g.L_k * 4 : 0);
+  w.fr_ctl = (int32_t*)take(frame ? 256 : 0);
+  w.fr_attn_ws = take(frame ? fc::attention_tc_workspace_bytes() : 0);
   w.total = off;
   return w;
 }
@@ -295,7 +317,7 @@ int make_geom(const fc_score_desc* d, ScoreGeom& g) {
   g.H_q = d->H_q; g.H_kv = d->H_kv; g.d = d->d; g.L_q = d->L_q; g.L_k = d->L_k;
   g.group = d->H_q / d->H_kv;
   g.n_q = g.group * d->L_q;
-  if (g.n_q > 128) return FC_ERR_UNSUPPORTED;
+  if (g.n_q > kCoreMaxQueries && (g.group != 1 || g.L_q > fc::kScoreFrameMaxQueries)) return FC_ERR_UNSUPPORTED;
   g.n_tiles = (d->L_k + kTile - 1) / kTile;
   g.n_partials = g.n_tiles;
   g.q_hs = d->q_hs; g.q_rs = d->q_rs; g.k_hs = d->k_hs; g.k_rs = d->k_rs;
@@ -319,8 +341,56 @@ int run(cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, co
   score_mean_key_kernel<<<g.H_kv, 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
   FC_LAUNCH_CHECK("score_mean_key_kernel");
   float* imp_buf = imp ? imp : w.imp_tmp;
-  score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, w.S, w.lse, w.mean_key, imp_accum, phase,
+  score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, w.S, w.lse, w.mean_key, nullptr, imp_accum, phase,
                                                    n_steps, imp_buf, w.a, w.a_partial);
+  FC_LAUNCH_CHECK("score_pass2_kernel");
+  if (phase != 1) {
+    score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
+    FC_LAUNCH_CHECK("score_finalize_kernel");
+  }
+  return FC_OK;
+}
+
+// Frame-level pipeline (bf16, one query head per key head, any number of queries up to kScoreFrameMaxQueries).
+template <int D>
+int run_frame(fc_ctx* ctx, cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, const void* K,
+              float* imp_accum, int phase, int n_steps, float* imp, float* red, float* score, uint32_t* status) {
+  using T = __nv_bfloat16;
+  dim3 grid(g.n_tiles, g.H_kv);
+  // 1. sums of normalised keys per tile (no queries: the logit loop of the kernel is empty)
+  ScoreGeom g0 = g;
+  g0.n_q = 0;
+  const size_t smem1 = (size_t)kTile * (D + 1) * 4;
+  FC_CUDA_CHECK(cudaFuncSetAttribute(score_pass1_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1));
+  score_pass1_kernel<T, D><<<grid, kTile, smem1, st>>>((const T*)Q, (const T*)K, g0, nullptr, w.mk_partial);
+  FC_LAUNCH_CHECK("score_pass1_kernel");
+  score_mean_key_kernel<<<g.H_kv, 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
+  FC_LAUNCH_CHECK("score_mean_key_kernel");
+  // 2. log-sum-exp of every query over the candidates: one chunk of L_q rows that sees all L_k keys; V = K
+  FC_CUDA_CHECK(cudaMemsetAsync(w.fr_ctl, 0, 8, st));                // active_ids[0] = 0
+  FC_CUDA_CHECK(cudaMemsetAsync((char*)w.fr_ctl + 4, 1, 1, st));     // n_active = 1 (little-endian)
+  fc::AttnGeom a;
+  a.H_q = g.H_kv; a.H_kv = g.H_kv; a.d = g.d; a.W = 1; a.group = 1; a.n_seg = 1;
+  a.q_hs = g.q_hs; a.q_rs = g.q_rs; a.k_hs = g.k_hs; a.k_rs = g.k_rs; a.v_hs = g.k_hs; a.v_rs = g.k_rs;
+  a.o_hs = (int64_t)g.L_q * g.d; a.o_rs = g.d; a.kv_rows = g.L_k; a.lse_hs = g.L_q; a.tok_hs = 0;
+  a.scale = g.scale;
+  a.q_row_off[0] = 0; a.q_row_off[1] = g.L_q;
+  a.vis[0] = g.L_k;
+  a.seg_log[0] = 0; a.seg_log[1] = g.L_k; a.seg_phys[0] = 0;
+  a.tok_index = nullptr;
+  a.active_ids = w.fr_ctl; a.n_active = w.fr_ctl + 1;
+  a.lse = w.lse;
+  a.status = status;
+  int rc = fc::attention_tc(ctx, st, a, Q, K, K, w.fr_O, w.fr_attn_ws, fc::attention_tc_workspace_bytes(), false);
+  if (rc != FC_OK) return rc;
+  // 3. attention mass of every key
+  rc = fc::score_frame_mass(ctx, st, g.H_kv, g.d, g.L_q, g.L_k, g.scale * 1.4426950408889634f, Q, g.q_hs, g.q_rs, K,
+                            g.k_hs, g.k_rs, w.lse, w.fr_mass, status);
+  if (rc != FC_OK) return rc;
+  // 4. mean over the queries, accumulation over steps, redundancy logits; 5. finalize
+  float* imp_buf = imp ? imp : w.imp_tmp;
+  score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, nullptr, nullptr, w.mean_key, w.fr_mass, imp_accum,
+                                                   phase, n_steps, imp_buf, w.a, w.a_partial);
   FC_LAUNCH_CHECK("score_pass2_kernel");
   if (phase != 1) {
     score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
@@ -359,6 +429,11 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
   if (!fc::aligned16(ws)) return FC_ERR_MISALIGNED;
   cudaStream_t st = (cudaStream_t)stream;
   if (desc->impl < 0 || desc->impl > 2) return FC_ERR_INVALID_ARG;
+  if (g.n_q > kCoreMaxQueries) {
+    if (dtype != FC_BF16 || desc->impl == 1) return FC_ERR_UNSUPPORTED;
+    if (g.d == 128) return run_frame<128>(ctx, st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score, status);
+    return run_frame<64>(ctx, st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score, status);
+  }
   const bool tc_ok = dtype == FC_BF16 && g.group == 1 && g.L_q <= fc::kScoreTcMaxQueries - 2;
   if (desc->impl == 2 && !tc_ok) return FC_ERR_UNSUPPORTED;
   if (tc_ok && desc->impl != 1) {

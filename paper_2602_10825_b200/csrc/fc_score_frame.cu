@@ -1,0 +1,192 @@
+// Attention mass of every candidate key under many observation queries (a latent frame or a whole chunk of
+// them) on tcgen05 tensor cores: the importance of Eq. 9 at frame-level query granularity, where the score stage
+// is a dense contraction instead of a streaming read.
+//
+//   mass[h, j] = sum_i exp(q_i . k_j * scale - lse_i)        lse_i = log sum_j exp(q_i . k_j * scale)
+//
+// lse comes from the caller (the chunk-attention kernel run over exactly the candidates emits it).  The logits
+// are recomputed here, not stored: S[key, query] = K Q^T, one key row per thread, so that the sum over the
+// queries stays inside a thread.  A CTA owns one (head, tile of 128 keys): the key tile is loaded once, the
+// head's query tiles stream through a 2-stage TMA ring (they stay in L2: every CTA of the head reads them), one
+// thread issues the MMAs into two 128-column accumulators and four warps turn them into masses.  Two CTAs share
+// an SM (2 x 256 tensor-memory columns, 2 x 97 KiB of shared memory; one CTA when the head has more than about
+// 3000 queries, whose log-sum-exps sit in shared memory), which puts two exponentiating warps on every
+// scheduler: the special-function unit, 16 exponentials per clock, is what bounds the kernel.
+// Sums are fixed-order: results are bit-reproducible from run to run.  Every mbarrier wait is bounded.
+#include <cmath>
+
+#include "fc_attention.cuh"
+#include "fc_score.cuh"
+#include "fc_tcgen05.cuh"
+#include "fc_tcgen05_ld.cuh"
+
+namespace {
+
+using namespace fc::sm100;
+
+constexpr int kKeys = 128, kQueries = 128;  // tile: MMA M and N
+constexpr int kQRing = 2;
+constexpr int kThreads = 192;  // warps 0-3 masses, warp 4 copies, warp 5 MMAs
+
+struct MassSmem {
+  uint64_t k_full, q_full[kQRing], q_free[kQRing], s_full[2], s_free[2];
+  uint32_t tmem_base, abort;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 2)
+score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, int L_q,
+                  int L_k, float scale_log2, const float* __restrict__ lse, int64_t lse_hs,
+                  float* __restrict__ mass, uint32_t* __restrict__ status) {
+  constexpr uint32_t kTileBytes = kKeys * D * 2;
+  constexpr int kAtoms = D / 64;
+  constexpr uint32_t kAtomBytes = kKeys * 128;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t k_s = smem_u32(smem), q_s = k_s + kTileBytes;
+  MassSmem* sh = (MassSmem*)(smem + (1 + kQRing) * kTileBytes);
+  // minus the log-sum-exp of every query of the head in the log2 domain, padded to whole tiles with -inf
+  float* nlse_s = (float*)(sh + 1);
+  volatile uint32_t* abort = &sh->abort;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int hk = blockIdx.y, tile = blockIdx.x;
+  const int n_qt = (L_q + kQueries - 1) / kQueries;
+
+  if (tid == 0) {
+    mbar_init(smem_u32(&sh->k_full), 1);
+    for (int s = 0; s < kQRing; ++s) {
+      mbar_init(smem_u32(&sh->q_full[s]), 1);
+      mbar_init(smem_u32(&sh->q_free[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sh->s_full[b]), 1);
+      mbar_init(smem_u32(&sh->s_free[b]), 4);  // warps 0-3
+    }
+    mbar_fence_init();
+    sh->abort = 0;
+    tma_prefetch_desc(&tmap_q);
+    tma_prefetch_desc(&tmap_k);
+  }
+  for (int i = tid; i < n_qt * kQueries; i += kThreads)
+    nlse_s[i] = i < L_q ? -lse[(int64_t)hk * lse_hs + i] * 1.4426950408889634f : -INFINITY;
+  if (warp == 0) {
+    tmem_alloc(smem_u32(&sh->tmem_base), 2 * kQueries);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sh->tmem_base;
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ copies
+    if (lane == 0) {
+      mbar_expect_tx(smem_u32(&sh->k_full), kTileBytes);
+      for (int x = 0; x < kAtoms; ++x)
+        tma_load_3d(k_s + x * kAtomBytes, &tmap_k, smem_u32(&sh->k_full), x * 64, tile * kKeys, hk);
+      for (int t = 0; t < n_qt; ++t) {
+        const int st = t % kQRing, ph = (t / kQRing) & 1;
+        if (!mbar_wait_bounded(smem_u32(&sh->q_free[st]), ph ^ 1, abort)) break;
+        mbar_expect_tx(smem_u32(&sh->q_full[st]), kTileBytes);
+        for (int x = 0; x < kAtoms; ++x)
+          tma_load_3d(q_s + st * kTileBytes + x * kAtomBytes, &tmap_q, smem_u32(&sh->q_full[st]), x * 64, t * kQueries,
+                      hk);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------------------------------------------ MMAs: S[key, query] = K Q^T
+    if (lane == 0) {
+      constexpr uint32_t kIdesc = idesc_bf16_f32(kKeys, kQueries, false, false);
+      const uint64_t dk = smem_desc_sw128(k_s, 16, 1024), dq = smem_desc_sw128(q_s, 16, 1024);
+      mbar_wait_bounded(smem_u32(&sh->k_full), 0, abort);
+      for (int t = 0; t < n_qt; ++t) {
+        const int st = t % kQRing, ph = (t / kQRing) & 1, b = t & 1;
+        if (!mbar_wait_bounded(smem_u32(&sh->q_full[st]), ph, abort)) break;
+        if (!mbar_wait_bounded(smem_u32(&sh->s_free[b]), ((t >> 1) & 1) ^ 1, abort)) break;
+        tc_fence_after();
+        const uint64_t b0 = dq + (uint64_t)(st * (kTileBytes >> 4));
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
+          umma_ss(tmem + b * kQueries, dk + off, b0 + off, kIdesc, kk > 0);
+        }
+        umma_commit(smem_u32(&sh->s_full[b]));
+        umma_commit(smem_u32(&sh->q_free[st]));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ masses: one key row per thread
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const uint64_t sc2 = pack2(scale_log2, scale_log2);
+    uint64_t acc[2] = {0ull, 0ull};
+    for (int t = 0; t < n_qt; ++t) {
+      const int b = t & 1;
+      if (!mbar_wait_bounded(smem_u32(&sh->s_full[b]), (t >> 1) & 1, abort)) break;
+      tc_fence_after();
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t sv[64];
+        tmem_ld64_wait(tmem + lane_base + b * kQueries + half * 64, sv);
+        const float2* nl = reinterpret_cast<const float2*>(nlse_s + t * kQueries + half * 64);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float2 n2 = nl[i];  // the same address in every lane: a broadcast
+          const uint64_t x =
+              fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sc2, pack2(n2.x, n2.y));
+          float x0, x1;
+          unpack2(x, x0, x1);
+          acc[i & 1] = add2(acc[i & 1], pack2(ex2(x0), ex2(x1)));  // padding queries: ex2(-inf) = 0
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
+    }
+    float a0, a1, a2, a3;
+    unpack2(acc[0], a0, a1);
+    unpack2(acc[1], a2, a3);
+    const int j = tile * kKeys + warp * 32 + lane;
+    if (j < L_k) mass[(int64_t)hk * L_k + j] = (a0 + a1) + (a2 + a3);
+  }
+
+  if (*abort) {
+    // something never arrived: give copies and instructions still in flight time to land before the
+    // shared and tensor memory of this CTA are handed back
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (tid == 0 && *abort && status) atomicOr(status, FC_DEV_TIMEOUT);
+  if (warp == 0) tmem_dealloc(tmem, 2 * kQueries);
+}
+
+}  // namespace
+
+namespace fc {
+
+int score_frame_mass(fc_ctx* ctx, cudaStream_t st, int H, int d, int L_q, int L_k, float scale_log2, const void* Q,
+                     int64_t q_hs, int64_t q_rs, const void* K, int64_t k_hs, int64_t k_rs, const float* lse,
+                     float* mass, uint32_t* status) {
+  if (L_q > kScoreFrameMaxQueries) return FC_ERR_UNSUPPORTED;
+  CUtensorMap tq, tk;
+  int rc;
+  if ((rc = make_tmap(ctx, &tq, Q, d, L_q, H, q_rs, H > 1 ? q_hs : q_rs * L_q)) != FC_OK) return rc;
+  if ((rc = make_tmap(ctx, &tk, K, d, L_k, H, k_rs, H > 1 ? k_hs : k_rs * L_k)) != FC_OK) return rc;
+  const int n_qt = (L_q + kQueries - 1) / kQueries;
+  // at least 97 KiB, so that a third CTA (and its 256 columns) never joins the SM
+  const size_t need = (1 + kQRing) * (size_t)kKeys * d * 2 + sizeof(MassSmem) + (size_t)n_qt * kQueries * 4 + 1024;
+  const size_t smem = std::max<size_t>(need, 97 * 1024);
+  if (smem > 227 * 1024) return FC_ERR_UNSUPPORTED;  // above 113 KiB one CTA per SM instead of two
+  dim3 grid((L_k + kKeys - 1) / kKeys, H);
+  if (d == 128) {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(score_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    score_mass_kernel<128><<<grid, kThreads, smem, st>>>(tq, tk, L_q, L_k, scale_log2, lse, (int64_t)L_q, mass, status);
+  } else {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(score_mass_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    score_mass_kernel<64><<<grid, kThreads, smem, st>>>(tq, tk, L_q, L_k, scale_log2, lse, (int64_t)L_q, mass, status);
+  }
+  FC_LAUNCH_CHECK("score_mass_kernel");
+  return FC_OK;
+}
+
+}  // namespace fc

@@ -338,6 +338,32 @@ def test_score_tensor_core_matches_cuda_core_full_size(ctx):
     assert np.abs(b.double().cpu().numpy() - want).max() <= 1e-4 * np.abs(want).max()
 
 
+@pytest.mark.parametrize("d,L_q,L_k", [(128, 300, 1000), (64, 129, 700), (128, 1560, 2345)])
+def test_score_frame_level_queries(ctx, d, L_q, L_k):
+    # frame-level query granularity: more observation queries than the token-level pipelines take (two full
+    # query tiles and a ragged one; one query past a tile; a whole latent frame), ragged key tiles, a zero key
+    Q = wl.normal((2, L_q, d), 61, 0.7, torch.bfloat16)
+    K = wl.normal((2, L_k, d), 62, 0.7, torch.bfloat16)
+    K[1, 5] = 0
+    _score_case(ctx, Q, K, 0.07, 7)
+
+
+def test_score_frame_level_accumulated_over_steps(ctx):
+    K = wl.normal((2, 900, 128), 71, 0.5, torch.bfloat16)
+    Qs = [wl.normal((2, 200, 128), 72 + s, 0.5, torch.bfloat16) for s in range(2)]
+    acc_o = np.zeros((2, 900), np.float64)
+    acc_g = torch.zeros((2, 900), device="cuda")
+    for s, q in enumerate(Qs):
+        phase = 2 if s == 1 else 1
+        want = oracle.kv_score(wl.bits(q), wl.bits(K), imp_accum=acc_o, accum_phase=phase, n_steps=2)
+        imp = torch.empty((2, 900), device="cuda")
+        got = ctx.kv_score(dev(q), dev(K), imp_accum=acc_g, accum_phase=phase, n_steps=2, imp=imp)
+    torch.cuda.synchronize()
+    np.testing.assert_allclose(imp.cpu().numpy(), want["imp"], rtol=0, atol=1e-4 * want["imp"].max())
+    np.testing.assert_allclose(got["score"].cpu().numpy(), want["score"], rtol=0,
+                               atol=1e-4 * np.abs(want["score"]).max())
+
+
 def test_score_gqa_and_d64(ctx):
     Q = wl.normal((4, 20, 64), 31, 1.0)
     K = wl.normal((2, 300, 64), 32, 1.0)

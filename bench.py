@@ -168,6 +168,25 @@ class DeviceStep:
                 events[i][1].record()
 
 
+def time_frame_score(step, iters=20):
+    """fc_kv_score with one latent frame of observation queries (30 x 52 tokens) instead of 50 tokens: the score
+    stage as a dense contraction.  Separate from the timed step; returns (ms per call, L_q)."""
+    L_q = min(1560, step.w.n_c)
+    R = step.Q.shape[1]
+    Q_frame = step.Q[:, R - L_q:]
+    score = torch.empty_like(step.score)
+    for _ in range(3):
+        step.ctx.kv_score(Q_frame, step.K_cand, lambda_=step.w.lam, pool_k=step.w.pool_k, score=score, status=step.status)
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record()
+    for _ in range(iters):
+        step.ctx.kv_score(Q_frame, step.K_cand, lambda_=step.w.lam, pool_k=step.w.pool_k, score=score, status=step.status)
+    t1.record()
+    torch.cuda.synchronize()
+    return t0.elapsed_time(t1) / iters, L_q
+
+
 def attention_flops(w, active):
     return w.attention_flops(active)
 
@@ -430,6 +449,16 @@ def main():
         if not args.no_e2e:
             line["e2e"] = {"value": job_throughput(world, flops, e2e_step_ms), "unit": "TFLOP/s",
                            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_step_ms}
+        if w.dtype == "bf16" and world == 1:
+            fr_ms, fr_lq = time_frame_score(step)
+            fr_flops = 2 * 2.0 * fr_lq * step.L_k * w.d * w.H  # the logits twice: log-sum-exp pass and mass pass
+            fr_tflops = fr_flops / (fr_ms * 1e-3) / 1e12
+            line["roofline_score_frame"] = {
+                "bound": "tensor", "achieved": fr_tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": fr_tflops / peaks["bf16_tflops"], "traffic": None, "ms": fr_ms, "L_q": fr_lq,
+                "kernel": "attention_ws_kernel (log-sum-exp pass) + score_mass_kernel + CUDA-core key statistics and "
+                          "finalize (whole fc_kv_score call, outside the timed step); algorithmic FLOPs = "
+                          "2 passes x 2 L_q L_k d H", "peak_kind": peak_kind + " burst"}
         if args.sweep:
             line["sweep"] = run_sweep(step, (0.05, 0.1, 0.2), 30, peaks["bf16_tflops"])
         if world == 1 and not args.no_cpu_baseline:

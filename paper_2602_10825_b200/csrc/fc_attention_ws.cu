@@ -92,25 +92,6 @@ struct Item {
   bool b_valid;  // tile B has at least one row of the chunk (false for the ragged last item of a chunk)
 };
 
-// 2^x for a pair of values on the fma pipe: x = n + r with n = round(x) (the low mantissa bits of x + 1.5 * 2^23)
-// and r in [-0.5, 0.5]; 2^r by a cubic (relative error 7.5e-5, a thirtieth of a bf16 rounding step), 2^n by
-// adding n to the exponent field.  x is clamped at -125 so that the exponent field cannot wrap.
-__device__ __forceinline__ void ex2_fma_pair(uint64_t x, float& p0, float& p1) {
-  float x0, x1;
-  unpack2(x, x0, x1);
-  const uint64_t xc = pack2(fmaxf(x0, -125.f), fmaxf(x1, -125.f));
-  const uint64_t t = add2(xc, pack2(12582912.f, 12582912.f));
-  const uint64_t r = add2(xc, fma2(t, pack2(-1.f, -1.f), pack2(12582912.f, 12582912.f)));  // x - (t - magic)
-  uint64_t q = fma2(pack2(0.0551716648f, 0.0551716648f), r, pack2(0.2426111251f, 0.2426111251f));
-  q = fma2(q, r, pack2(0.6932609677f, 0.6932609677f));
-  q = fma2(q, r, pack2(0.9999280572f, 0.9999280572f));
-  float t0, t1, q0, q1;
-  unpack2(t, t0, t1);
-  unpack2(q, q0, q1);
-  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23));
-  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23));
-}
-
 // P = 2^(S * scale - m) for one row of a 64-column half tile, written as bf16 to tensor-memory columns
 // [t_p, t_p + 32); returns the row sum.
 __device__ __forceinline__ float exp_half(const uint32_t (&sv)[kHalf], float scale_log2, float m, uint32_t t_p) {

@@ -6,7 +6,9 @@
 //
 // lse comes from the caller (the chunk-attention kernel run over exactly the candidates emits it).  The logits
 // are recomputed here, not stored: S[key, query] = K Q^T, one key row per thread, so that the sum over the
-// queries stays inside a thread.  A CTA owns one (head, tile of 128 keys): the key tile is loaded once, the
+// queries stays inside a thread.  A CTA owns one head and every gridDim.x-th tile of 128 keys of it (set-up, the
+// head's log-sum-exps in shared memory and the tensor-memory allocation are paid once per CTA); per key tile the
+// keys are loaded once and the
 // head's query tiles stream through a 2-stage TMA ring (they stay in L2: every CTA of the head reads them), one
 // thread issues the MMAs into two 128-column accumulators and four warps turn them into masses.  Two CTAs share
 // an SM (2 x 256 tensor-memory columns, 2 x 97 KiB of shared memory; one CTA when the head has more than about
@@ -29,7 +31,7 @@ constexpr int kQRing = 2;
 constexpr int kThreads = 192;  // warps 0-3 masses, warp 4 copies, warp 5 MMAs
 
 struct MassSmem {
-  uint64_t k_full, q_full[kQRing], q_free[kQRing], s_full[2], s_free[2];
+  uint64_t k_full, k_free, q_full[kQRing], q_free[kQRing], s_full[2], s_free[2];
   uint32_t tmem_base, abort;
 };
 
@@ -49,11 +51,12 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   float* nlse_s = (float*)(sh + 1);
   volatile uint32_t* abort = &sh->abort;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int hk = blockIdx.y, tile = blockIdx.x;
-  const int n_qt = (L_q + kQueries - 1) / kQueries;
+  const int hk = blockIdx.y;
+  const int n_qt = (L_q + kQueries - 1) / kQueries, n_kt = (L_k + kKeys - 1) / kKeys;
 
   if (tid == 0) {
     mbar_init(smem_u32(&sh->k_full), 1);
+    mbar_init(smem_u32(&sh->k_free), 1);
     for (int s = 0; s < kQRing; ++s) {
       mbar_init(smem_u32(&sh->q_full[s]), 1);
       mbar_init(smem_u32(&sh->q_free[s]), 1);
@@ -81,16 +84,20 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   if (warp == 4) {
     // ------------------------------------------------------------------ copies
     if (lane == 0) {
-      mbar_expect_tx(smem_u32(&sh->k_full), kTileBytes);
-      for (int x = 0; x < kAtoms; ++x)
-        tma_load_3d(k_s + x * kAtomBytes, &tmap_k, smem_u32(&sh->k_full), x * 64, tile * kKeys, hk);
-      for (int t = 0; t < n_qt; ++t) {
-        const int st = t % kQRing, ph = (t / kQRing) & 1;
-        if (!mbar_wait_bounded(smem_u32(&sh->q_free[st]), ph ^ 1, abort)) break;
-        mbar_expect_tx(smem_u32(&sh->q_full[st]), kTileBytes);
+      uint32_t tq = 0, it = 0;  // query tiles and key tiles loaded so far (ring phases)
+      for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x, ++it) {
+        if (!mbar_wait_bounded(smem_u32(&sh->k_free), (it & 1) ^ 1, abort)) break;
+        mbar_expect_tx(smem_u32(&sh->k_full), kTileBytes);
         for (int x = 0; x < kAtoms; ++x)
-          tma_load_3d(q_s + st * kTileBytes + x * kAtomBytes, &tmap_q, smem_u32(&sh->q_full[st]), x * 64, t * kQueries,
-                      hk);
+          tma_load_3d(k_s + x * kAtomBytes, &tmap_k, smem_u32(&sh->k_full), x * 64, tile * kKeys, hk);
+        for (int t = 0; t < n_qt; ++t, ++tq) {
+          const int st = tq % kQRing, ph = (tq / kQRing) & 1;
+          if (!mbar_wait_bounded(smem_u32(&sh->q_free[st]), ph ^ 1, abort)) break;
+          mbar_expect_tx(smem_u32(&sh->q_full[st]), kTileBytes);
+          for (int x = 0; x < kAtoms; ++x)
+            tma_load_3d(q_s + st * kTileBytes + x * kAtomBytes, &tmap_q, smem_u32(&sh->q_full[st]), x * 64,
+                        t * kQueries, hk);
+        }
       }
     }
   } else if (warp == 5) {
@@ -98,30 +105,36 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     if (lane == 0) {
       constexpr uint32_t kIdesc = idesc_bf16_f32(kKeys, kQueries, false, false);
       const uint64_t dk = smem_desc_sw128(k_s, 16, 1024), dq = smem_desc_sw128(q_s, 16, 1024);
-      mbar_wait_bounded(smem_u32(&sh->k_full), 0, abort);
-      for (int t = 0; t < n_qt; ++t) {
-        const int st = t % kQRing, ph = (t / kQRing) & 1, b = t & 1;
-        if (!mbar_wait_bounded(smem_u32(&sh->q_full[st]), ph, abort)) break;
-        if (!mbar_wait_bounded(smem_u32(&sh->s_free[b]), ((t >> 1) & 1) ^ 1, abort)) break;
-        tc_fence_after();
-        const uint64_t b0 = dq + (uint64_t)(st * (kTileBytes >> 4));
+      uint32_t tq = 0, it = 0;
+      for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x, ++it) {
+        if (!mbar_wait_bounded(smem_u32(&sh->k_full), it & 1, abort)) break;
+        for (int t = 0; t < n_qt; ++t, ++tq) {
+          const int st = tq % kQRing, ph = (tq / kQRing) & 1, b = tq & 1;
+          if (!mbar_wait_bounded(smem_u32(&sh->q_full[st]), ph, abort)) break;
+          if (!mbar_wait_bounded(smem_u32(&sh->s_free[b]), ((tq >> 1) & 1) ^ 1, abort)) break;
+          tc_fence_after();
+          const uint64_t b0 = dq + (uint64_t)(st * (kTileBytes >> 4));
 #pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
-          umma_ss(tmem + b * kQueries, dk + off, b0 + off, kIdesc, kk > 0);
+          for (int kk = 0; kk < D / 16; ++kk) {
+            const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
+            umma_ss(tmem + b * kQueries, dk + off, b0 + off, kIdesc, kk > 0);
+          }
+          umma_commit(smem_u32(&sh->s_full[b]));
+          umma_commit(smem_u32(&sh->q_free[st]));
         }
-        umma_commit(smem_u32(&sh->s_full[b]));
-        umma_commit(smem_u32(&sh->q_free[st]));
+        umma_commit(smem_u32(&sh->k_free));  // the key tile has been read by every MMA issued for it
       }
     }
   } else {
     // ------------------------------------------------------------------ masses: one key row per thread
     const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
     const uint64_t sc2 = pack2(scale_log2, scale_log2);
+    uint32_t tq = 0;
+    for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x) {
     uint64_t acc[2] = {0ull, 0ull};
-    for (int t = 0; t < n_qt; ++t) {
-      const int b = t & 1;
-      if (!mbar_wait_bounded(smem_u32(&sh->s_full[b]), (t >> 1) & 1, abort)) break;
+    for (int t = 0; t < n_qt; ++t, ++tq) {
+      const int b = tq & 1;
+      if (!mbar_wait_bounded(smem_u32(&sh->s_full[b]), (tq >> 1) & 1, abort)) break;
       tc_fence_after();
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
@@ -133,9 +146,16 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
           const float2 n2 = nl[i];  // the same address in every lane: a broadcast
           const uint64_t x =
               fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sc2, pack2(n2.x, n2.y));
-          float x0, x1;
-          unpack2(x, x0, x1);
-          acc[i & 1] = add2(acc[i & 1], pack2(ex2(x0), ex2(x1)));  // padding queries: ex2(-inf) = 0
+          float p0, p1;
+          if ((i & 3) == 3) {
+            ex2_fma_pair(x, p0, p1);  // one pair in four on the fma pipe: the special-function unit is the bound
+          } else {
+            float x0, x1;
+            unpack2(x, x0, x1);
+            p0 = ex2(x0);
+            p1 = ex2(x1);
+          }
+          acc[i & 1] = add2(acc[i & 1], pack2(p0, p1));  // padding queries: 2^-inf = 0 (2^-125 on the fma pipe)
         }
       }
       tc_fence_before();
@@ -147,6 +167,7 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     unpack2(acc[1], a2, a3);
     const int j = tile * kKeys + warp * 32 + lane;
     if (j < L_k) mass[(int64_t)hk * L_k + j] = (a0 + a1) + (a2 + a3);
+    }
   }
 
   if (*abort) {
@@ -177,7 +198,10 @@ int score_frame_mass(fc_ctx* ctx, cudaStream_t st, int H, int d, int L_q, int L_
   const size_t need = (1 + kQRing) * (size_t)kKeys * d * 2 + sizeof(MassSmem) + (size_t)n_qt * kQueries * 4 + 1024;
   const size_t smem = std::max<size_t>(need, 97 * 1024);
   if (smem > 227 * 1024) return FC_ERR_UNSUPPORTED;  // above 113 KiB one CTA per SM instead of two
-  dim3 grid((L_k + kKeys - 1) / kKeys, H);
+  // two CTAs per SM over all heads; every CTA stays inside one head
+  const int n_kt = (L_k + kKeys - 1) / kKeys;
+  const int per_sm = smem <= 113 * 1024 ? 2 : 1;
+  dim3 grid(std::max(1, std::min(n_kt, (per_sm * ctx->sm_count) / H)), H);
   if (d == 128) {
     FC_CUDA_CHECK(cudaFuncSetAttribute(score_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     score_mass_kernel<128><<<grid, kThreads, smem, st>>>(tq, tk, L_q, L_k, scale_log2, lse, (int64_t)L_q, mass, status);

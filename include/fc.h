@@ -193,9 +193,15 @@ int fc_chunk_attention(fc_ctx* ctx, void* stream, const fc_attn_desc* desc, cons
  * of the l2-normalised keys with a zeroed diagonal (Eq. 11), evaluated through the mean-key
  * identity of the paper's efficiency appendix, column mean_j = (mean_i khat_i).khat_j -
  * |khat_j|^2 / L_k, with khat = k / max(|k|, 1e-12); Score = lambda*Imp~ - (1-lambda)*Red (Eq. 12).
+ *
+ * Query granularity (the paper's ablation of token / frame / chunk observation queries): up to
+ * 128 query rows per kv head take the streaming pipelines (the paper's setting, the last 50
+ * tokens); more than that - a latent frame or a whole chunk of queries, bf16, H_q == H_kv, up
+ * to 8192 - take the frame-level pipeline, in which both passes over the logits run on the
+ * tensor cores.
  */
 typedef struct {
-  int32_t H_q, H_kv, d, L_q, L_k;  /* L_q * (H_q/H_kv) <= 128 */
+  int32_t H_q, H_kv, d, L_q, L_k;  /* L_q * (H_q/H_kv) <= 128, or bf16 with H_q == H_kv and L_q <= 8192 */
   int64_t q_hs, q_rs, k_hs, k_rs;  /* element strides */
   float scale;                     /* 0 => 1/sqrt(d) */
   float lambda;                    /* mixing coefficient (paper: 0.07) */

@@ -141,3 +141,57 @@ def test_denoising_sweep_decisions_and_attention_of_the_active_chunks(ctx, eps):
                     assert torch.equal(O[:, q_off[c]:q_off[c + 1]].cpu(), O0[:, q_off[c]:q_off[c + 1]])
     assert min_margin > 1e-3 * eps, f"a step came within {min_margin} of eps; change the seed"
     assert fractions[0] == 1.0 and fractions[-1] <= 0.5 and min(fractions) < max(fractions)
+
+
+@pytest.mark.parametrize("eps", [0.1, 0.15])
+def test_blocks_at_staggered_noise_levels(ctx, eps):
+    # the second model family in small: five blocks in flight, block i two denoising steps behind block i - 1, four
+    # warm-up steps per block (so at any step some blocks are forced, some decide by threshold), a clean overlap
+    # region in front; decisions bit-exact at every step, attention of the active blocks at three of them
+    full = wl.CONFIGS["skyreels_bf16"]
+    w = wl.Workload("blocks_small", "bf16", H=2, d=full.d, W=full.W, n_c=344, B=344, L_k=688, seed=full.seed,
+                    sigma=full.sigma, D=192, eps=eps, warmup_m=full.warmup_m)
+    n_el = w.n_c * w.hidden
+    off = np.arange(w.W + 1, dtype=np.int64) * n_el
+    Q, K, V = wl.qkv(w)
+    q_off, vis, slo, spo = wl.prefix_layout(w)
+    Qg, Kg, Vg = Q.cuda(), K.cuda(), V.cuda()
+    O0 = wl.normal((w.H, w.window_rows, w.d), 78, 1.0, torch.bfloat16)
+    acc_o = np.zeros(w.W, np.float32)
+    acc_g = torch.zeros(w.W, device="cuda")
+    n_steps, lag = 14, 2
+    n_forced = n_reused = 0
+    for s in range(n_steps):
+        step = np.maximum(s - lag * np.arange(w.W), 0).astype(np.int32)
+        target = wl.uniform((w.W,), 900 + s, 0.0, 0.12).numpy()
+        for _ in range(8):  # guard band around the threshold, as in the sweep test
+            cur, prev = wl.indicator_pair(w.W, n_el, target, 6000 + s)
+            want = oracle.chunk_decide(wl.bits(cur), wl.bits(prev), off, step, w.warmup_m, eps, acc_o)
+            margin = np.abs(acc_o + want["l1rel"] - eps)[step >= w.warmup_m]
+            if margin.size == 0 or margin.min() > 1e-3 * eps:
+                break
+            target = target * 1.03
+        assert margin.size == 0 or margin.min() > 1e-3 * eps
+        got = ctx.chunk_decide(cur.cuda(), prev.cuda(), off, i32(step), w.warmup_m, eps, acc_g)
+        torch.cuda.synchronize()
+        assert got["recompute"].cpu().numpy().tolist() == want["recompute"].tolist(), f"step {s}"
+        assert got["active_ids"].cpu().numpy()[:want["n_active"]].tolist() == want["active_ids"].tolist()
+        acc_o = want["acc"]
+        active = want["active_ids"].tolist()
+        n_forced += int((step < w.warmup_m).sum())
+        n_reused += w.W - len(active)
+        assert all(c in active for c in range(w.W) if step[c] < w.warmup_m)  # warm-up blocks always compute
+        if s in (3, 8, 13):
+            O = O0.cuda().clone()
+            ctx.chunk_attention(Qg, Kg, Vg, q_off, vis, slo, spo, got["active_ids"], got["n_active"], O)
+            torch.cuda.synchronize()
+            rows = wl.sample_rows(w, 16, s)
+            rows = rows[np.isin(rows // w.n_c, active)]
+            if len(rows):
+                O_want, _ = oracle.chunk_attention(wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, slo, spo, active,
+                                                   sample_rows=rows)
+                _check_attention(O.double().cpu().numpy()[:, rows], O_want)
+            for c in range(w.W):
+                if c not in active:
+                    assert torch.equal(O[:, q_off[c]:q_off[c + 1]].cpu(), O0[:, q_off[c]:q_off[c + 1]])
+    assert n_forced > 0 and n_reused > 0

@@ -7,7 +7,9 @@ from it.  Every tensor comes from a ``torch.Generator`` on the CPU with a fixed
 seed and is rounded once to its storage dtype; the same bits go to both sides.
 
 Shapes follow the paper's models: hidden width 3072 = 24 heads x 128, chunks
-of 3-4 latent frames of 30 x 52 patches, cache budgets of 4-8 chunks.
+of 3-4 latent frames of 30 x 52 patches, cache budgets of 4-8 chunks; for the
+second model family hidden width 1536 = 12 heads x 128 and blocks of 5 latent
+frames of 34 x 60 patches.
 """
 from __future__ import annotations
 
@@ -74,6 +76,12 @@ CONFIGS = {
                                L_k=32760, seed=3, sigma=0.5, keys="ar1", n_steps=4),
     "sweep_bf16": Workload("sweep_bf16", "bf16", H=24, d=128, W=16, n_c=6240, B=37440,
                            L_k=43680, seed=4, sigma=0.5, n_steps=30),
+    # The paper's second model family: blocks inside a chunk at staggered noise levels.  A "chunk" of the
+    # library is one block here: 5 latent frames of 34 x 60 patches (540P), 12 heads x 128 (hidden 1536); five
+    # blocks in flight; the clean region is the 17-frame (5 latent frames) overlap with the previous chunk;
+    # thresholds 0.1 / 0.15, four warm-up steps.
+    "skyreels_bf16": Workload("skyreels_bf16", "bf16", H=12, d=128, W=5, n_c=10200, B=10200,
+                              L_k=20400, seed=5, sigma=0.5, eps=0.1, warmup_m=4, n_steps=50),
 }
 
 

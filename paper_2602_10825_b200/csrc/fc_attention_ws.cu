@@ -59,11 +59,6 @@ constexpr float kRescaleThreshold = 8.f;  // log2 units
 #endif
 static_assert(256 * FC_ATTN_REGS_HI + 128 * FC_ATTN_REGS_LO <= 384 * 168, "register split exceeds the CTA's pool");
 static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg takes multiples of 8");
-// exponentiate against the running reference before the tile's maximum is known (see the softmax loop)
-#ifndef FC_ATTN_SPECULATE
-#define FC_ATTN_SPECULATE 1
-#endif
-constexpr bool kSpeculate = FC_ATTN_SPECULATE != 0;
 // of every four column pairs, how many take their exponential on the fma pipe instead of the special-function unit
 #ifndef FC_ATTN_POLY_OF_4
 #define FC_ATTN_POLY_OF_4 1
@@ -545,46 +540,26 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
               }
               return fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
             };
-            float alpha = 1.f, row_sum;
-            if (kSpeculate && !first && mine_valid == kHalf) {
-              // Common case: the reference maximum of the row does not move (it moves only when a half tile exceeds
-              // it by 2^8).  So exponentiate against the reference at once, without looking for the maximum first.
-              // A row whose sum stays below 2^8 cannot hold a term above 2^8; only if some row of the warp
-              // exceeds that is the maximum computed, and the half tile redone for the rows that have to move.
-              row_sum = exp_half(sv, scale_log2, m, t_su);
-              if (__any_sync(0xffffffffu, !(row_sum <= 256.f))) {  // 2^kRescaleThreshold; also catches inf / NaN
-                const float tile_max = row_max();
-                const bool move = tile_max > m + kRescaleThreshold;
-                if (__any_sync(0xffffffffu, move)) {
-                  if (move) {
-                    alpha = ex2(m - tile_max);
-                    m = tile_max;
-                  }
-                  tmem_wait_st();
-                  wait_pv();
-                  rescale_o(alpha);
-                  row_sum = exp_half(sv, scale_log2, m, t_su);
-                }
-              }
-            } else {
-              if (mine_valid < kHalf) {
+            if (mine_valid < kHalf) {
 #pragma unroll
-                for (int i = 0; i < kHalf; ++i)
-                  if (i >= mine_valid) sv[i] = 0xff800000u;  // -inf
-              }
-              const float tile_max = row_max();  // -inf if the half holds no visible token: then nothing moves
-              // lazy reference update: move only when the maximum grew by more than the threshold
-              const bool move = tile_max > m + kRescaleThreshold;  // always true on an item's first half (m = -inf)
-              if (move) {
-                alpha = ex2(m - tile_max);
-                m = tile_max;
-              }
-              if (!first && __any_sync(0xffffffffu, move)) {
-                wait_pv();
-                rescale_o(alpha);
-              }
-              row_sum = exp_half(sv, scale_log2, m, t_su);  // masked columns: ex2(-inf) = 0 exactly
+              for (int i = 0; i < kHalf; ++i)
+                if (i >= mine_valid) sv[i] = 0xff800000u;  // -inf
             }
+            const float tile_max = row_max();  // -inf if the half holds no visible token: then nothing moves
+            // Lazy reference update: move only when the maximum grew by more than the threshold.  Either way the
+            // exponent below is at most 2^kRescaleThreshold, which is what lets a share of the exponentials run on
+            // the fma pipe (ex2_fma_pair has no upper clamp).
+            const bool move = tile_max > m + kRescaleThreshold;  // always true on an item's first half (m = -inf)
+            float alpha = 1.f;
+            if (move) {
+              alpha = ex2(m - tile_max);
+              m = tile_max;
+            }
+            if (!first && __any_sync(0xffffffffu, move)) {
+              wait_pv();
+              rescale_o(alpha);
+            }
+            const float row_sum = exp_half(sv, scale_log2, m, t_su);  // masked columns: 2^-inf = 0 (2^-125 on the fma pipe)
             l = l * alpha + row_sum;
             tmem_wait_st();
             tc_fence_before();

@@ -214,7 +214,10 @@ __device__ __forceinline__ float ex2(float x) {
 }
 // 2^x for a pair of values on the fma pipe: x = n + r with n = round(x) (the low mantissa bits of x + 1.5 * 2^23)
 // and r in [-0.5, 0.5]; 2^r by a cubic (relative error 7.5e-5, a thirtieth of a bf16 rounding step), 2^n by
-// adding n to the exponent field.  x is clamped at -125 so that the exponent field cannot wrap.
+// adding n to the exponent field.  x is clamped at -125 from below (the result is then 2^-125 instead of 0).
+// PRECONDITION: x <= 127.  Above that the exponent field wraps and the result is garbage of either sign, so
+// callers use this only where x is bounded by construction (a softmax argument after its reference maximum is
+// known).
 __device__ __forceinline__ void ex2_fma_pair(uint64_t x, float& p0, float& p1) {
   float x0, x1;
   unpack2(x, x0, x1);

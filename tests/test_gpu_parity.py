@@ -386,6 +386,36 @@ def test_score_accumulated_over_steps(ctx):
                                atol=1e-4 * np.abs(want["score"]).max())
 
 
+def test_attention_logit_jump_far_above_the_running_maximum(ctx):
+    # Keys late in the prefix whose logits exceed everything before them by hundreds of log2 units, for single query
+    # rows only (the other rows of the warp see nothing unusual): the reference maximum must move for exactly those
+    # rows and O be rescaled, whichever unit takes the exponential of that column (columns 6 and 7 of a 64-column
+    # half go to the fma pipe, columns 0 and 64 to the special-function unit).
+    w = wl.Workload("jump", "bf16", H=2, d=128, W=1, n_c=256, B=1536, L_k=0, seed=91, sigma=0.5)
+    Q, K, V = wl.qkv(w)
+    Q[:, :, 120:] = 0
+    K[:, :, 120:] = 0
+    for n, (pos, row) in enumerate(((128 * 5 + 6, 0), (128 * 7 + 71, 37), (128 * 9 + 64, 130), (128 * 11 + 7, 255))):
+        Q[:, row, 120 + n] = 8.0           # only this row has a component along axis 120 + n ...
+        K[:, pos, 120 + n] = 200.0 * (n + 1)  # ... and only this key: logit 1600 (n+1) / sqrt(128) = 141 (n+1) nats
+    q_off, vis, slo, spo = wl.prefix_layout(w)
+    O = torch.zeros_like(Q).cuda()
+    lse = torch.empty((w.H, w.n_c), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.chunk_attention(dev(Q), dev(K), dev(V), q_off, vis, slo, spo, i32([0]), i32([1]), O, lse=lse, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    O_want, lse_want = oracle.chunk_attention(wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, slo, spo, [0])
+    got = O.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - O_want).max() <= 1e-2
+    assert np.linalg.norm(got - O_want) <= 1e-2 * np.linalg.norm(O_want)
+    np.testing.assert_allclose(lse.double().cpu().numpy(), lse_want, rtol=1e-5, atol=2e-3)
+    # the four rows attend to their own key alone
+    for pos, row in ((128 * 5 + 6, 0), (128 * 7 + 71, 37), (128 * 9 + 64, 130), (128 * 11 + 7, 255)):
+        assert np.abs(got[:, row] - V[:, pos].double().numpy()).max() <= 1e-2
+
+
 # ------------------------------------------------------------------------------------ select + compact
 
 def _select_case(ctx, score, B, K=None, V=None):

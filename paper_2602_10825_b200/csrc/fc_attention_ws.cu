@@ -15,10 +15,10 @@
 // its own "full" and "P ready" barriers, and P (bf16) of a half overwrites the first 32 columns of that half.
 // The order of one MMA thread is S0(0) S1(0) | PV0(0) S0(1) PV1(0) S1(1) | PV0(1) S0(2) ..., so the S of the
 // next key tile's first half is issued as soon as P of this tile's first half has been handed to the tensor pipe,
-// while the softmax is still busy with the second half.  A softmax warp therefore finds its next half already
-// computed and never waits for a round trip through the tensor pipe: what bounds it is the special-function
-// unit (2 tiles x 128 x 128 exponentials at 16 per clock = 2048 clocks per pair of tiles, the same as the
-// tensor pipe's 2048).  With whole-tile S accumulators the chain S -> softmax -> PV -> S of one tile was the
+// while the softmax is still busy with the second half.  A softmax warp therefore normally finds its next half
+// already computed instead of waiting for a round trip through the tensor pipe; what bounds it then is the
+// special-function unit (2 tiles x 128 x 128 exponentials at 16 per clock = 2048 clocks per pair of tiles, the
+// same as the tensor pipe's 2048).  With whole-tile S accumulators the chain S -> softmax -> PV -> S of one tile was the
 // critical path (about 3800 clocks per pair of tiles, measured).  The price: an S instruction with N = 64 reads
 // the whole 128-row Q operand from shared memory for half the columns and takes about 45 clocks instead of 32
 // (measured), so the tensor pipe needs about 1240 clocks per tile instead of 1024.

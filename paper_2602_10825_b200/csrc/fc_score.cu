@@ -6,9 +6,9 @@
 // kernel below; everything else (fp32, grouped query heads, more queries) takes the
 // CUDA-core pipeline (below).  bf16 inputs with more than 128 observation queries per key head (a latent frame
 // or a whole chunk of them) take the frame-level pipeline: key norms and mean key by the CUDA-core pass-1 kernel
-// without queries, every query's log-sum-exp over the candidates by the chunk-attention kernel (its LSE output;
-// its O output goes to scratch), the attention mass by the tensor-core kernel of fc_score_frame.cu, then the
-// CUDA-core pass-2 kernel fed with that mass, and the finalize kernel.
+// without queries, every query's log-sum-exp over the candidates and then the attention mass of every key by the
+// tensor-core kernel of fc_score_frame.cu (two launches), then the CUDA-core pass-2 kernel fed with that mass, and
+// the finalize kernel.
 // The CUDA-core pipeline, five launches per call:
 //   pass1     one thread per key: raw logits of all observation queries against its key,
 //             written to the workspace; normalised key summed per 128-key tile (mean key)
@@ -20,7 +20,6 @@
 //   finalize  softmax of a over the head, max-pool of the importance, lambda-mix
 #include <cmath>
 
-#include "fc_attention.cuh"
 #include "fc_common.cuh"
 #include "fc_score.cuh"
 
@@ -274,10 +273,8 @@ struct ScoreWs {
   float* tc_lse2;
   float* tc_norm2;
   // frame-level path
-  void* fr_O;          // scratch output of the attention launch that produces the log-sum-exps
   float* fr_mass;      // [H, L_k] sum over the queries of exp(logit - lse)
-  int32_t* fr_ctl;     // active_ids[1] = 0, n_active = 1
-  void* fr_attn_ws;
+  float2* fr_ml;       // [H, slices, L_q] (maximum, sum) of every query over a slice of the keys
   size_t total;
 };
 
@@ -301,10 +298,8 @@ ScoreWs carve(const ScoreGeom& g, void* ws) {
   w.tc_colsum = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * g.d * 4);
   w.tc_lse2 = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxQueries * 4);
   w.tc_norm2 = (float*)take((size_t)g.H_kv * g.L_k * 4);
-  w.fr_O = take(frame ? (size_t)g.H_kv * g.L_q * g.d * 2 : 0);
   w.fr_mass = (float*)take(frame ? (size_t)g.H_kv * g.L_k * 4 : 0);
-  w.fr_ctl = (int32_t*)take(frame ? 256 : 0);
-  w.fr_attn_ws = take(frame ? fc::attention_tc_workspace_bytes() : 0);
+  w.fr_ml = (float2*)take(frame ? (size_t)g.H_kv * fc::kScoreFrameMaxSlices * g.L_q * 8 : 0);
   w.total = off;
   return w;
 }
@@ -366,26 +361,9 @@ int run_frame(fc_ctx* ctx, cudaStream_t st, const ScoreGeom& g, const ScoreWs& w
   FC_LAUNCH_CHECK("score_pass1_kernel");
   score_mean_key_kernel<<<g.H_kv, 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
   FC_LAUNCH_CHECK("score_mean_key_kernel");
-  // 2. log-sum-exp of every query over the candidates: one chunk of L_q rows that sees all L_k keys; V = K
-  FC_CUDA_CHECK(cudaMemsetAsync(w.fr_ctl, 0, 8, st));                // active_ids[0] = 0
-  FC_CUDA_CHECK(cudaMemsetAsync((char*)w.fr_ctl + 4, 1, 1, st));     // n_active = 1 (little-endian)
-  fc::AttnGeom a;
-  a.H_q = g.H_kv; a.H_kv = g.H_kv; a.d = g.d; a.W = 1; a.group = 1; a.n_seg = 1;
-  a.q_hs = g.q_hs; a.q_rs = g.q_rs; a.k_hs = g.k_hs; a.k_rs = g.k_rs; a.v_hs = g.k_hs; a.v_rs = g.k_rs;
-  a.o_hs = (int64_t)g.L_q * g.d; a.o_rs = g.d; a.kv_rows = g.L_k; a.lse_hs = g.L_q; a.tok_hs = 0;
-  a.scale = g.scale;
-  a.q_row_off[0] = 0; a.q_row_off[1] = g.L_q;
-  a.vis[0] = g.L_k;
-  a.seg_log[0] = 0; a.seg_log[1] = g.L_k; a.seg_phys[0] = 0;
-  a.tok_index = nullptr;
-  a.active_ids = w.fr_ctl; a.n_active = w.fr_ctl + 1;
-  a.lse = w.lse;
-  a.status = status;
-  int rc = fc::attention_tc(ctx, st, a, Q, K, K, w.fr_O, w.fr_attn_ws, fc::attention_tc_workspace_bytes(), false);
-  if (rc != FC_OK) return rc;
-  // 3. attention mass of every key
-  rc = fc::score_frame_mass(ctx, st, g.H_kv, g.d, g.L_q, g.L_k, g.scale * 1.4426950408889634f, Q, g.q_hs, g.q_rs, K,
-                            g.k_hs, g.k_rs, w.lse, w.fr_mass, status);
+  // 2., 3. log-sum-exp of every query over the candidates, then the attention mass of every key
+  int rc = fc::score_frame_mass(ctx, st, g.H_kv, g.d, g.L_q, g.L_k, g.scale * 1.4426950408889634f, Q, g.q_hs, g.q_rs, K,
+                                g.k_hs, g.k_rs, w.fr_ml, w.lse, w.fr_mass, status);
   if (rc != FC_OK) return rc;
   // 4. mean over the queries, accumulation over steps, redundancy logits; 5. finalize
   float* imp_buf = imp ? imp : w.imp_tmp;

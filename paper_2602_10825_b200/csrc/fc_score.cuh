@@ -11,6 +11,7 @@ constexpr int kScoreTcMaxQueries = 64;  // query rows of the tensor-core path: o
                                         // padded) and two rows for the mean key
 constexpr int kScoreTcMaxSlices = 64;   // slices of key tiles per head
 constexpr int kScoreFrameMaxQueries = 8192;  // observation queries of the frame-level path
+constexpr int kScoreFrameMaxSlices = 16;     // slices of the key range in its row-statistics launch
 
 struct ScoreTcArgs {
   int H, L_q, L_k, n_tiles, tiles_per_slice, n_slices;  // n_tiles = ceil(L_k / 128); slices are set by score_tc_run
@@ -30,10 +31,12 @@ struct ScoreTcArgs {
 int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs args, int d, int64_t q_hs, int64_t q_rs, int64_t k_hs,
                  int64_t k_rs, const void* Q, const void* K);
 
-// Frame-level query granularity: mass[h, j] = sum_i exp(q_i . k_j * scale - lse[h, i]) on tensor cores
-// (bf16, one query head per key head); `lse` [H, L_q] natural-log, `mass` [H, L_k], both dense.
+// Frame-level query granularity on tensor cores (bf16, one query head per key head): first every query's (maximum,
+// sum) over slices of the candidates into `ml_part` ([H, kScoreFrameMaxSlices, L_q] at most, log2 domain), their
+// merge into `nlse` ([H, L_q], minus the log2-domain log-sum-exp), then mass[h, j] = sum_i exp(q_i . k_j * scale -
+// lse[h, i]) ([H, L_k] dense).
 int score_frame_mass(fc_ctx* ctx, cudaStream_t st, int H, int d, int L_q, int L_k, float scale_log2, const void* Q,
-                     int64_t q_hs, int64_t q_rs, const void* K, int64_t k_hs, int64_t k_rs, const float* lse,
+                     int64_t q_hs, int64_t q_rs, const void* K, int64_t k_hs, int64_t k_rs, float2* ml_part, float* nlse,
                      float* mass, uint32_t* status);
 
 }  // namespace fc

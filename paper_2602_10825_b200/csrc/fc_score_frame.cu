@@ -4,9 +4,12 @@
 //
 //   mass[h, j] = sum_i exp(q_i . k_j * scale - lse_i)        lse_i = log sum_j exp(q_i . k_j * scale)
 //
-// lse comes from the caller (the chunk-attention kernel run over exactly the candidates emits it).  The logits
-// are recomputed here, not stored: S[key, query] = K Q^T, one key row per thread, so that the sum over the
-// queries stays inside a thread.  A CTA owns one head and every gridDim.x-th tile of 128 keys of it (set-up, the
+// Two launches of one kernel, which recomputes the logits instead of storing them and picks the orientation whose
+// reduction stays inside a thread:
+//   row statistics   S[query, key] = Q K^T, one query row per thread: running (max, sum) over all keys -> lse
+//   masses           S[key, query] = K Q^T, one key row per thread: the sum over the queries
+// Below, the tile that a CTA holds is the "own" tile (queries for the statistics, keys for the masses) and the
+// other operand streams past it.  A CTA owns one head and every gridDim.x-th tile of 128 keys of it (set-up, the
 // head's log-sum-exps in shared memory and the tensor-memory allocation are paid once per CTA); per key tile the
 // keys are loaded once and the
 // head's query tiles stream through a 2-stage TMA ring (they stay in L2: every CTA of the head reads them), one
@@ -35,10 +38,29 @@ struct MassSmem {
   uint32_t tmem_base, abort;
 };
 
-template <int D>
+// kStats = true:  own = queries, stream = keys, gridDim.z slices of the key range; out = ml_out [H, slices, L_q]:
+//                 (reference maximum, sum against it) of every query over the slice, log2 domain
+// kStats = false: own = keys, stream = queries (gridDim.z = 1); out = mass [H, L_k]; nlse_in [H, L_q] = minus every
+//                 query's log-sum-exp in the log2 domain (score_frame_lse_kernel merges the slices)
+// In the code below tmap_k / L_k / "key tile" name the OWN operand and tmap_q / L_q / "query tile" the STREAMED one.
+// minus the log2-domain log-sum-exp of every query: the slices' (maximum, sum) pairs merged in slice order
+__global__ void score_frame_lse_kernel(const float2* __restrict__ ml, int n_slices, int L_q, float* __restrict__ nlse) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x, hk = blockIdx.y;
+  if (i >= L_q) return;
+  float m = -INFINITY, l = 0.f;
+  for (int sl = 0; sl < n_slices; ++sl) {
+    const float2 p = ml[((int64_t)hk * n_slices + sl) * L_q + i];
+    const float mn = fmaxf(m, p.x);
+    l = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * exp2f(p.x - mn));
+    m = mn;
+  }
+  nlse[(int64_t)hk * L_q + i] = -(m + log2f(l));
+}
+
+template <int D, bool kStats>
 __global__ void __launch_bounds__(kThreads, 2)
 score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, int L_q,
-                  int L_k, float scale_log2, const float* __restrict__ lse, int64_t lse_hs,
+                  int L_k, float scale_log2, const float* __restrict__ nlse_in, float2* __restrict__ ml_out,
                   float* __restrict__ mass, uint32_t* __restrict__ status) {
   constexpr uint32_t kTileBytes = kKeys * D * 2;
   constexpr int kAtoms = D / 64;
@@ -53,6 +75,9 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int hk = blockIdx.y;
   const int n_qt = (L_q + kQueries - 1) / kQueries, n_kt = (L_k + kKeys - 1) / kKeys;
+  // streamed tiles of this CTA (a slice of them in the statistics launch)
+  const int per_slice = (n_qt + (int)gridDim.z - 1) / (int)gridDim.z;
+  const int t_begin = blockIdx.z * per_slice, t_end = min(n_qt, t_begin + per_slice);
 
   if (tid == 0) {
     mbar_init(smem_u32(&sh->k_full), 1);
@@ -70,8 +95,10 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
   }
-  for (int i = tid; i < n_qt * kQueries; i += kThreads)
-    nlse_s[i] = i < L_q ? -lse[(int64_t)hk * lse_hs + i] * 1.4426950408889634f : -INFINITY;
+  if (!kStats) {
+    for (int i = tid; i < n_qt * kQueries; i += kThreads)
+      nlse_s[i] = i < L_q ? nlse_in[(int64_t)hk * L_q + i] : -INFINITY;  // padding queries: 2^-inf = 0
+  }
   if (warp == 0) {
     tmem_alloc(smem_u32(&sh->tmem_base), 2 * kQueries);
     tmem_relinquish();
@@ -90,7 +117,7 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         mbar_expect_tx(smem_u32(&sh->k_full), kTileBytes);
         for (int x = 0; x < kAtoms; ++x)
           tma_load_3d(k_s + x * kAtomBytes, &tmap_k, smem_u32(&sh->k_full), x * 64, tile * kKeys, hk);
-        for (int t = 0; t < n_qt; ++t, ++tq) {
+        for (int t = t_begin; t < t_end; ++t, ++tq) {
           const int st = tq % kQRing, ph = (tq / kQRing) & 1;
           if (!mbar_wait_bounded(smem_u32(&sh->q_free[st]), ph ^ 1, abort)) break;
           mbar_expect_tx(smem_u32(&sh->q_full[st]), kTileBytes);
@@ -108,7 +135,7 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       uint32_t tq = 0, it = 0;
       for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x, ++it) {
         if (!mbar_wait_bounded(smem_u32(&sh->k_full), it & 1, abort)) break;
-        for (int t = 0; t < n_qt; ++t, ++tq) {
+        for (int t = t_begin; t < t_end; ++t, ++tq) {
           const int st = tq % kQRing, ph = (tq / kQRing) & 1, b = tq & 1;
           if (!mbar_wait_bounded(smem_u32(&sh->q_full[st]), ph, abort)) break;
           if (!mbar_wait_bounded(smem_u32(&sh->s_free[b]), ((tq >> 1) & 1) ^ 1, abort)) break;
@@ -132,10 +159,58 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     uint32_t tq = 0;
     for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x) {
     uint64_t acc[2] = {0ull, 0ull};
-    for (int t = 0; t < n_qt; ++t, ++tq) {
+    float m_run = -INFINITY, l_run = 0.f;  // kStats: running reference maximum (log2 domain) and sum against it
+    for (int t = t_begin; t < t_end; ++t, ++tq) {
       const int b = tq & 1;
       if (!mbar_wait_bounded(smem_u32(&sh->s_full[b]), (tq >> 1) & 1, abort)) break;
       tc_fence_after();
+      if constexpr (kStats) {
+        // one query row against 128 keys: the reference moves only when the tile maximum exceeds it by 2^8, so
+        // the exponents stay below 2^8 and the sum is rescaled a few times per row at most
+        const int cols_valid = min(kQueries, L_q - t * kQueries);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          uint32_t sv[64];
+          tmem_ld64_wait(tmem + lane_base + b * kQueries + half * 64, sv);
+          if (cols_valid < half * 64 + 64) {
+#pragma unroll
+            for (int i = 0; i < 64; ++i)
+              if (half * 64 + i >= cols_valid) sv[i] = 0xff800000u;  // -inf
+          }
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+          for (int i = 0; i < 64; i += 8) {
+#pragma unroll
+            for (int c4 = 0; c4 < 4; ++c4)
+              mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
+          }
+          const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
+          if (tile_max > m_run + 8.f) {
+            l_run *= ex2(m_run - tile_max);  // 0 on the first tile (m_run = -inf)
+            m_run = tile_max;
+          }
+          const uint64_t nm2 = pack2(-m_run, -m_run);
+          uint64_t sum2[2] = {0ull, 0ull};
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const uint64_t x = fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sc2, nm2);
+            float p0, p1;
+            if ((i & 3) == 3) {
+              ex2_fma_pair(x, p0, p1);  // x <= 8 here
+            } else {
+              float x0, x1;
+              unpack2(x, x0, x1);
+              p0 = ex2(x0);
+              p1 = ex2(x1);
+            }
+            sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
+          }
+          float a0, a1, a2, a3;
+          unpack2(sum2[0], a0, a1);
+          unpack2(sum2[1], a2, a3);
+          l_run += (a0 + a1) + (a2 + a3);
+        }
+      } else {
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t sv[64];
@@ -158,6 +233,7 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
           acc[i & 1] = add2(acc[i & 1], pack2(p0, p1));  // padding queries: 2^-inf = 0 (2^-125 on the fma pipe)
         }
       }
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
@@ -166,7 +242,12 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
     unpack2(acc[0], a0, a1);
     unpack2(acc[1], a2, a3);
     const int j = tile * kKeys + warp * 32 + lane;
-    if (j < L_k) mass[(int64_t)hk * L_k + j] = (a0 + a1) + (a2 + a3);
+    if (j < L_k) {
+      if constexpr (kStats)
+        ml_out[((int64_t)hk * gridDim.z + blockIdx.z) * L_k + j] = make_float2(m_run, l_run);
+      else
+        mass[(int64_t)hk * L_k + j] = (a0 + a1) + (a2 + a3);
+    }
     }
   }
 
@@ -185,32 +266,62 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
 
 namespace fc {
 
+namespace {
+template <int D, bool kStats>
+int launch(fc_ctx* ctx, cudaStream_t st, const CUtensorMap& t_stream, const CUtensorMap& t_own, int H, int n_stream,
+           int n_own, float scale_log2, const float* nlse, float2* ml, int n_slices, float* mass, uint32_t* status) {
+  const int n_st = (n_stream + kQueries - 1) / kQueries, n_ot = (n_own + kKeys - 1) / kKeys;
+  // at least 97 KiB, so that a third CTA (and its 256 columns) never joins the SM
+  const size_t need = (1 + kQRing) * (size_t)kKeys * D * 2 + sizeof(MassSmem) + (kStats ? 0 : (size_t)n_st * kQueries * 4) + 1024;
+  const size_t smem = std::max<size_t>(need, 97 * 1024);
+  if (smem > 227 * 1024) return FC_ERR_UNSUPPORTED;  // above 113 KiB one CTA per SM instead of two
+  // two CTAs per SM over all heads; every CTA stays inside one head
+  const int per_sm = smem <= 113 * 1024 ? 2 : 1;
+  dim3 grid(std::max(1, std::min(n_ot, (per_sm * ctx->sm_count) / H)), H, kStats ? n_slices : 1);
+  FC_CUDA_CHECK(cudaFuncSetAttribute(score_mass_kernel<D, kStats>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  score_mass_kernel<D, kStats><<<grid, kThreads, smem, st>>>(t_stream, t_own, n_stream, n_own, scale_log2, nlse, ml, mass,
+                                                             status);
+  FC_LAUNCH_CHECK("score_mass_kernel");
+  return FC_OK;
+}
+}  // namespace
+
+int score_frame_slices(fc_ctx* ctx, int H, int L_q, int L_k) {
+  // Slices of the key range in the statistics launch: with few query tiles per head the (head, query tile) pairs
+  // alone do not fill the CTA slots evenly.  Cost model: waves of CTAs x (key tiles per slice + 3 tiles' worth of
+  // set-up per CTA).
+  const int n_qt = (L_q + kKeys - 1) / kKeys, n_kt = (L_k + kQueries - 1) / kQueries, slots = 2 * ctx->sm_count;
+  int best = 1;
+  int64_t best_cost = INT64_MAX;
+  for (int sl = 1; sl <= kScoreFrameMaxSlices && sl <= n_kt; ++sl) {
+    const int64_t ctas = (int64_t)std::min(n_qt, std::max(1, slots / H)) * H * sl;
+    const int64_t own_per_cta = (n_qt + std::max(1, slots / H) - 1) / std::max(1, slots / H);
+    const int64_t cost = ((ctas + slots - 1) / slots) * own_per_cta * ((n_kt + sl - 1) / sl + 3);
+    if (cost < best_cost) {
+      best_cost = cost;
+      best = sl;
+    }
+  }
+  return best;
+}
+
 int score_frame_mass(fc_ctx* ctx, cudaStream_t st, int H, int d, int L_q, int L_k, float scale_log2, const void* Q,
-                     int64_t q_hs, int64_t q_rs, const void* K, int64_t k_hs, int64_t k_rs, const float* lse,
+                     int64_t q_hs, int64_t q_rs, const void* K, int64_t k_hs, int64_t k_rs, float2* ml_part, float* nlse,
                      float* mass, uint32_t* status) {
   if (L_q > kScoreFrameMaxQueries) return FC_ERR_UNSUPPORTED;
   CUtensorMap tq, tk;
   int rc;
   if ((rc = make_tmap(ctx, &tq, Q, d, L_q, H, q_rs, H > 1 ? q_hs : q_rs * L_q)) != FC_OK) return rc;
   if ((rc = make_tmap(ctx, &tk, K, d, L_k, H, k_rs, H > 1 ? k_hs : k_rs * L_k)) != FC_OK) return rc;
-  const int n_qt = (L_q + kQueries - 1) / kQueries;
-  // at least 97 KiB, so that a third CTA (and its 256 columns) never joins the SM
-  const size_t need = (1 + kQRing) * (size_t)kKeys * d * 2 + sizeof(MassSmem) + (size_t)n_qt * kQueries * 4 + 1024;
-  const size_t smem = std::max<size_t>(need, 97 * 1024);
-  if (smem > 227 * 1024) return FC_ERR_UNSUPPORTED;  // above 113 KiB one CTA per SM instead of two
-  // two CTAs per SM over all heads; every CTA stays inside one head
-  const int n_kt = (L_k + kKeys - 1) / kKeys;
-  const int per_sm = smem <= 113 * 1024 ? 2 : 1;
-  dim3 grid(std::max(1, std::min(n_kt, (per_sm * ctx->sm_count) / H)), H);
-  if (d == 128) {
-    FC_CUDA_CHECK(cudaFuncSetAttribute(score_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    score_mass_kernel<128><<<grid, kThreads, smem, st>>>(tq, tk, L_q, L_k, scale_log2, lse, (int64_t)L_q, mass, status);
-  } else {
-    FC_CUDA_CHECK(cudaFuncSetAttribute(score_mass_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    score_mass_kernel<64><<<grid, kThreads, smem, st>>>(tq, tk, L_q, L_k, scale_log2, lse, (int64_t)L_q, mass, status);
-  }
-  FC_LAUNCH_CHECK("score_mass_kernel");
-  return FC_OK;
+  const int n_slices = score_frame_slices(ctx, H, L_q, L_k);
+  // (max, sum) of every query over the slices of the candidates, their merge, then the mass of every key
+  if (d == 128) rc = launch<128, true>(ctx, st, tk, tq, H, L_k, L_q, scale_log2, nullptr, ml_part, n_slices, nullptr, status);
+  else rc = launch<64, true>(ctx, st, tk, tq, H, L_k, L_q, scale_log2, nullptr, ml_part, n_slices, nullptr, status);
+  if (rc != FC_OK) return rc;
+  score_frame_lse_kernel<<<dim3((L_q + 255) / 256, H), 256, 0, st>>>(ml_part, n_slices, L_q, nlse);
+  FC_LAUNCH_CHECK("score_frame_lse_kernel");
+  if (d == 128) return launch<128, false>(ctx, st, tq, tk, H, L_q, L_k, scale_log2, nlse, nullptr, 1, mass, status);
+  return launch<64, false>(ctx, st, tq, tk, H, L_q, L_k, scale_log2, nlse, nullptr, 1, mass, status);
 }
 
 }  // namespace fc

@@ -494,7 +494,7 @@ def main():
             line["roofline_score_frame"] = {
                 "bound": "tensor", "achieved": fr_tflops, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": fr_tflops / peaks["bf16_tflops"], "traffic": None, "ms": fr_ms, "L_q": fr_lq,
-                "kernel": "attention_ws_kernel (log-sum-exp pass) + score_mass_kernel + CUDA-core key statistics and "
+                "kernel": "score_mass_kernel x2 (row statistics, masses) + CUDA-core key statistics and "
                           "finalize (whole fc_kv_score call, outside the timed step); algorithmic FLOPs = "
                           "2 passes x 2 L_q L_k d H", "peak_kind": peak_kind + " burst"}
         if args.sweep:

@@ -30,19 +30,21 @@ namespace {
 using namespace fc::sm100;
 
 constexpr int kKeys = 128, kQueries = 128;  // tile: MMA M and N
-constexpr int kQRing = 2;
-constexpr int kThreads = 192;  // warps 0-3 masses, warp 4 copies, warp 5 MMAs
+constexpr int kRing = 4;     // streamed tiles in flight = logit accumulators in tensor memory (4 x 128 columns)
+#ifndef FC_FRAME_FMA_SHARE
+#define FC_FRAME_FMA_SHARE 1
+#endif
+constexpr int kFmaShare = FC_FRAME_FMA_SHARE;  // of every four column pairs, how many take their exponential on the fma pipe
+constexpr int kGroups = 4;   // consumer warpgroups; group g takes every fourth streamed tile
+constexpr int kThreads = 32 * (4 * kGroups + 2);  // 16 consumer warps, one copy warp, one MMA warp
 
 struct MassSmem {
-  uint64_t k_full, k_free, q_full[kQRing], q_free[kQRing], s_full[2], s_free[2];
+  uint64_t own_full[2], own_free[2], q_full[kRing], q_free[kRing], s_full[kRing], s_free[kRing];
+  uint64_t merge_bar;  // all consumer warps, once per own tile
   uint32_t tmem_base, abort;
+  float2 part[2][kGroups][kKeys];  // per own tile (double-buffered), group and row: partial mass or (maximum, sum)
 };
 
-// kStats = true:  own = queries, stream = keys, gridDim.z slices of the key range; out = ml_out [H, slices, L_q]:
-//                 (reference maximum, sum against it) of every query over the slice, log2 domain
-// kStats = false: own = keys, stream = queries (gridDim.z = 1); out = mass [H, L_k]; nlse_in [H, L_q] = minus every
-//                 query's log-sum-exp in the log2 domain (score_frame_lse_kernel merges the slices)
-// In the code below tmap_k / L_k / "key tile" name the OWN operand and tmap_q / L_q / "query tile" the STREAMED one.
 // minus the log2-domain log-sum-exp of every query: the slices' (maximum, sum) pairs merged in slice order
 __global__ void score_frame_lse_kernel(const float2* __restrict__ ml, int n_slices, int L_q, float* __restrict__ nlse) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x, hk = blockIdx.y;
@@ -58,7 +60,7 @@ __global__ void score_frame_lse_kernel(const float2* __restrict__ ml, int n_slic
 }
 
 template <int D, bool kStats>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k, int L_q,
                   int L_k, float scale_log2, const float* __restrict__ nlse_in, float2* __restrict__ ml_out,
                   float* __restrict__ mass, uint32_t* __restrict__ status) {
@@ -67,8 +69,8 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   constexpr uint32_t kAtomBytes = kKeys * 128;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const uint32_t k_s = smem_u32(smem), q_s = k_s + kTileBytes;
-  MassSmem* sh = (MassSmem*)(smem + (1 + kQRing) * kTileBytes);
+  const uint32_t k_s = smem_u32(smem), q_s = k_s + 2 * kTileBytes;  // own tiles (2), then the ring of streamed tiles
+  MassSmem* sh = (MassSmem*)(smem + (2 + kRing) * kTileBytes);
   // minus the log-sum-exp of every query of the head in the log2 domain, padded to whole tiles with -inf
   float* nlse_s = (float*)(sh + 1);
   volatile uint32_t* abort = &sh->abort;
@@ -80,16 +82,17 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   const int t_begin = blockIdx.z * per_slice, t_end = min(n_qt, t_begin + per_slice);
 
   if (tid == 0) {
-    mbar_init(smem_u32(&sh->k_full), 1);
-    mbar_init(smem_u32(&sh->k_free), 1);
-    for (int s = 0; s < kQRing; ++s) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&sh->own_full[s]), 1);
+      mbar_init(smem_u32(&sh->own_free[s]), 1);
+    }
+    for (int s = 0; s < kRing; ++s) {
       mbar_init(smem_u32(&sh->q_full[s]), 1);
       mbar_init(smem_u32(&sh->q_free[s]), 1);
+      mbar_init(smem_u32(&sh->s_full[s]), 1);
+      mbar_init(smem_u32(&sh->s_free[s]), 4);  // the four warps of the group that reads accumulator s
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sh->s_full[b]), 1);
-      mbar_init(smem_u32(&sh->s_free[b]), 4);  // warps 0-3
-    }
+    mbar_init(smem_u32(&sh->merge_bar), 4 * kGroups);
     mbar_fence_init();
     sh->abort = 0;
     tma_prefetch_desc(&tmap_q);
@@ -100,7 +103,7 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
       nlse_s[i] = i < L_q ? nlse_in[(int64_t)hk * L_q + i] : -INFINITY;  // padding queries: 2^-inf = 0
   }
   if (warp == 0) {
-    tmem_alloc(smem_u32(&sh->tmem_base), 2 * kQueries);
+    tmem_alloc(smem_u32(&sh->tmem_base), kRing * kQueries);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -108,17 +111,18 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   tc_fence_after();
   const uint32_t tmem = sh->tmem_base;
 
-  if (warp == 4) {
+  if (warp == 4 * kGroups) {
     // ------------------------------------------------------------------ copies
     if (lane == 0) {
-      uint32_t tq = 0, it = 0;  // query tiles and key tiles loaded so far (ring phases)
+      uint32_t tq = 0, it = 0;  // streamed tiles and own tiles loaded so far (ring phases)
       for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x, ++it) {
-        if (!mbar_wait_bounded(smem_u32(&sh->k_free), (it & 1) ^ 1, abort)) break;
-        mbar_expect_tx(smem_u32(&sh->k_full), kTileBytes);
+        const int o = it & 1;
+        if (!mbar_wait_bounded(smem_u32(&sh->own_free[o]), ((it >> 1) & 1) ^ 1, abort)) break;
+        mbar_expect_tx(smem_u32(&sh->own_full[o]), kTileBytes);
         for (int x = 0; x < kAtoms; ++x)
-          tma_load_3d(k_s + x * kAtomBytes, &tmap_k, smem_u32(&sh->k_full), x * 64, tile * kKeys, hk);
+          tma_load_3d(k_s + o * kTileBytes + x * kAtomBytes, &tmap_k, smem_u32(&sh->own_full[o]), x * 64, tile * kKeys, hk);
         for (int t = t_begin; t < t_end; ++t, ++tq) {
-          const int st = tq % kQRing, ph = (tq / kQRing) & 1;
+          const int st = tq % kRing, ph = (tq / kRing) & 1;
           if (!mbar_wait_bounded(smem_u32(&sh->q_free[st]), ph ^ 1, abort)) break;
           mbar_expect_tx(smem_u32(&sh->q_full[st]), kTileBytes);
           for (int x = 0; x < kAtoms; ++x)
@@ -127,127 +131,163 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
         }
       }
     }
-  } else if (warp == 5) {
-    // ------------------------------------------------------------------ MMAs: S[key, query] = K Q^T
+  } else if (warp == 4 * kGroups + 1) {
+    // ------------------------------------------------------------------ MMAs: S[own row, streamed row]
     if (lane == 0) {
       constexpr uint32_t kIdesc = idesc_bf16_f32(kKeys, kQueries, false, false);
+      constexpr int kSteps = D / 16;
       const uint64_t dk = smem_desc_sw128(k_s, 16, 1024), dq = smem_desc_sw128(q_s, 16, 1024);
+      // The issuing thread does not run ahead of the tensor pipe, so the operand descriptors of a tile are computed
+      // and pinned in registers before the waits, and its MMAs go out as one block of instructions.
+      uint64_t da[kSteps], db[kSteps];
       uint32_t tq = 0, it = 0;
       for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x, ++it) {
-        if (!mbar_wait_bounded(smem_u32(&sh->k_full), it & 1, abort)) break;
-        for (int t = t_begin; t < t_end; ++t, ++tq) {
-          const int st = tq % kQRing, ph = (tq / kQRing) & 1, b = tq & 1;
-          if (!mbar_wait_bounded(smem_u32(&sh->q_full[st]), ph, abort)) break;
-          if (!mbar_wait_bounded(smem_u32(&sh->s_free[b]), ((tq >> 1) & 1) ^ 1, abort)) break;
-          tc_fence_after();
-          const uint64_t b0 = dq + (uint64_t)(st * (kTileBytes >> 4));
+        const int o = it & 1;
 #pragma unroll
-          for (int kk = 0; kk < D / 16; ++kk) {
-            const uint64_t off = ((kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4;
-            umma_ss(tmem + b * kQueries, dk + off, b0 + off, kIdesc, kk > 0);
-          }
-          umma_commit(smem_u32(&sh->s_full[b]));
+        for (int kk = 0; kk < kSteps; ++kk)
+          da[kk] = dk + (uint64_t)((o * kTileBytes + (kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4);
+        pin(da);
+        if (!mbar_wait_bounded(smem_u32(&sh->own_full[o]), (it >> 1) & 1, abort)) break;
+        for (int t = t_begin; t < t_end; ++t, ++tq) {
+          const int st = tq % kRing, ph = (tq / kRing) & 1;  // ring slot = accumulator
+#pragma unroll
+          for (int kk = 0; kk < kSteps; ++kk)
+            db[kk] = dq + (uint64_t)((st * kTileBytes + (kk / 4) * kAtomBytes + (kk % 4) * 32) >> 4);
+          pin(db);
+          if (!mbar_wait_bounded(smem_u32(&sh->q_full[st]), ph, abort)) break;
+          if (!mbar_wait_bounded(smem_u32(&sh->s_free[st]), ph ^ 1, abort)) break;
+          tc_fence_after();
+          umma_ss_group<kSteps>(tmem + st * kQueries, da, db, kIdesc);
+          umma_commit(smem_u32(&sh->s_full[st]));
           umma_commit(smem_u32(&sh->q_free[st]));
         }
-        umma_commit(smem_u32(&sh->k_free));  // the key tile has been read by every MMA issued for it
+        umma_commit(smem_u32(&sh->own_free[o]));  // the own tile has been read by every MMA issued for it
       }
     }
   } else {
-    // ------------------------------------------------------------------ masses: one key row per thread
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    // ------------------------------------------------------------------ consumers: one own row per thread; group grp
+    // takes the streamed tiles whose ring slot is grp
+    const int grp = warp >> 2, quad = warp & 3;
+    const uint32_t t_acc = tmem + ((uint32_t)(quad * 32) << 16) + grp * kQueries;
     const uint64_t sc2 = pack2(scale_log2, scale_log2);
-    uint32_t tq = 0;
-    for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x) {
-    uint64_t acc[2] = {0ull, 0ull};
-    float m_run = -INFINITY, l_run = 0.f;  // kStats: running reference maximum (log2 domain) and sum against it
-    for (int t = t_begin; t < t_end; ++t, ++tq) {
-      const int b = tq & 1;
-      if (!mbar_wait_bounded(smem_u32(&sh->s_full[b]), (tq >> 1) & 1, abort)) break;
-      tc_fence_after();
-      if constexpr (kStats) {
-        // one query row against 128 keys: the reference moves only when the tile maximum exceeds it by 2^8, so
-        // the exponents stay below 2^8 and the sum is rescaled a few times per row at most
-        const int cols_valid = min(kQueries, L_q - t * kQueries);
+    const uint32_t b_sfull = smem_u32(&sh->s_full[grp]), b_sfree = smem_u32(&sh->s_free[grp]);
+    uint32_t tq = 0, it = 0;
+    for (int tile = blockIdx.x; tile < n_kt && !*abort; tile += gridDim.x, ++it) {
+      uint64_t acc[2] = {0ull, 0ull};
+      float m_run = -INFINITY, l_run = 0.f;  // kStats: running reference maximum (log2 domain) and sum against it
+      for (int t = t_begin; t < t_end; ++t, ++tq) {
+        if ((int)(tq % kRing) != grp) continue;
+        if (!mbar_wait_bounded(b_sfull, (tq / kRing) & 1, abort)) break;
+        tc_fence_after();
+        if constexpr (kStats) {
+          // one query row against 128 keys: the reference moves only when the tile maximum exceeds it by 2^8, so
+          // the exponents stay below 2^8 and the sum is rescaled a few times per row at most
+          const int cols_valid = min(kQueries, L_q - t * kQueries);
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          uint32_t sv[64];
-          tmem_ld64_wait(tmem + lane_base + b * kQueries + half * 64, sv);
-          if (cols_valid < half * 64 + 64) {
+          for (int half = 0; half < 2; ++half) {
+            uint32_t sv[64];
+            tmem_ld64_wait(t_acc + half * 64, sv);
+            if (cols_valid < half * 64 + 64) {
 #pragma unroll
-            for (int i = 0; i < 64; ++i)
-              if (half * 64 + i >= cols_valid) sv[i] = 0xff800000u;  // -inf
-          }
-          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-          for (int i = 0; i < 64; i += 8) {
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4)
-              mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
-          }
-          const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
-          if (tile_max > m_run + 8.f) {
-            l_run *= ex2(m_run - tile_max);  // 0 on the first tile (m_run = -inf)
-            m_run = tile_max;
-          }
-          const uint64_t nm2 = pack2(-m_run, -m_run);
-          uint64_t sum2[2] = {0ull, 0ull};
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const uint64_t x = fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sc2, nm2);
-            float p0, p1;
-            if ((i & 3) == 3) {
-              ex2_fma_pair(x, p0, p1);  // x <= 8 here
-            } else {
-              float x0, x1;
-              unpack2(x, x0, x1);
-              p0 = ex2(x0);
-              p1 = ex2(x1);
+              for (int i = 0; i < 64; ++i)
+                if (half * 64 + i >= cols_valid) sv[i] = 0xff800000u;  // -inf
             }
-            sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int i = 0; i < 64; i += 8) {
+#pragma unroll
+              for (int c4 = 0; c4 < 4; ++c4)
+                mx[c4] = max3(mx[c4], __uint_as_float(sv[i + 2 * c4]), __uint_as_float(sv[i + 2 * c4 + 1]));
+            }
+            const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
+            if (tile_max > m_run + 8.f) {
+              l_run *= ex2(m_run - tile_max);  // 0 on the first tile (m_run = -inf)
+              m_run = tile_max;
+            }
+            const uint64_t nm2 = pack2(-m_run, -m_run);
+            uint64_t sum2[2] = {0ull, 0ull};
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const uint64_t x = fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sc2, nm2);
+              float p0, p1;
+              if (kFmaShare > 0 && (i & 3) >= 4 - kFmaShare) {
+                ex2_fma_pair(x, p0, p1);  // x <= 8 here
+              } else {
+                float x0, x1;
+                unpack2(x, x0, x1);
+                p0 = ex2(x0);
+                p1 = ex2(x1);
+              }
+              sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
+            }
+            float a0, a1, a2, a3;
+            unpack2(sum2[0], a0, a1);
+            unpack2(sum2[1], a2, a3);
+            l_run += (a0 + a1) + (a2 + a3);
           }
-          float a0, a1, a2, a3;
-          unpack2(sum2[0], a0, a1);
-          unpack2(sum2[1], a2, a3);
-          l_run += (a0 + a1) + (a2 + a3);
+        } else {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            uint32_t sv[64];
+            tmem_ld64_wait(t_acc + half * 64, sv);
+            const float2* nl = reinterpret_cast<const float2*>(nlse_s + t * kQueries + half * 64);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float2 n2 = nl[i];  // the same address in every lane: a broadcast
+              const uint64_t x =
+                  fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sc2, pack2(n2.x, n2.y));
+              float p0, p1;
+              if (kFmaShare > 0 && (i & 3) >= 4 - kFmaShare) {
+                ex2_fma_pair(x, p0, p1);  // one pair in four on the fma pipe: the special-function unit is the bound
+              } else {
+                float x0, x1;
+                unpack2(x, x0, x1);
+                p0 = ex2(x0);
+                p1 = ex2(x1);
+              }
+              acc[i & 1] = add2(acc[i & 1], pack2(p0, p1));  // padding queries: 2^-inf = 0 (2^-125 on the fma pipe)
+            }
+          }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(b_sfree);
+      }
+      // the four groups' partial results of this own tile, merged by group 0 in group order
+      const int row = quad * 32 + lane;
+      if constexpr (kStats) {
+        sh->part[it & 1][grp][row] = make_float2(m_run, l_run);
       } else {
+        float a0, a1, a2, a3;
+        unpack2(acc[0], a0, a1);
+        unpack2(acc[1], a2, a3);
+        sh->part[it & 1][grp][row] = make_float2((a0 + a1) + (a2 + a3), 0.f);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sh->merge_bar));
+      // every consumer warp waits: no warp may arrive for the next own tile before this phase is complete
+      if (!mbar_wait_bounded(smem_u32(&sh->merge_bar), it & 1, abort)) break;
+      if (grp == 0) {
+        const int j = tile * kKeys + row;
+        if (j < L_k) {
+          if constexpr (kStats) {
+            float m = -INFINITY, l = 0.f;
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t sv[64];
-        tmem_ld64_wait(tmem + lane_base + b * kQueries + half * 64, sv);
-        const float2* nl = reinterpret_cast<const float2*>(nlse_s + t * kQueries + half * 64);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float2 n2 = nl[i];  // the same address in every lane: a broadcast
-          const uint64_t x =
-              fma2(pack2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), sc2, pack2(n2.x, n2.y));
-          float p0, p1;
-          if ((i & 3) == 3) {
-            ex2_fma_pair(x, p0, p1);  // one pair in four on the fma pipe: the special-function unit is the bound
+            for (int gq = 0; gq < kGroups; ++gq) {
+              const float2 p = sh->part[it & 1][gq][row];
+              const float mn = fmaxf(m, p.x);
+              l = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * exp2f(p.x - mn));
+              m = mn;
+            }
+            ml_out[((int64_t)hk * gridDim.z + blockIdx.z) * L_k + j] = make_float2(m, l);
           } else {
-            float x0, x1;
-            unpack2(x, x0, x1);
-            p0 = ex2(x0);
-            p1 = ex2(x1);
+            float sum = 0.f;
+#pragma unroll
+            for (int gq = 0; gq < kGroups; ++gq) sum += sh->part[it & 1][gq][row].x;
+            mass[(int64_t)hk * L_k + j] = sum;
           }
-          acc[i & 1] = add2(acc[i & 1], pack2(p0, p1));  // padding queries: 2^-inf = 0 (2^-125 on the fma pipe)
         }
       }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
-    }
-    float a0, a1, a2, a3;
-    unpack2(acc[0], a0, a1);
-    unpack2(acc[1], a2, a3);
-    const int j = tile * kKeys + warp * 32 + lane;
-    if (j < L_k) {
-      if constexpr (kStats)
-        ml_out[((int64_t)hk * gridDim.z + blockIdx.z) * L_k + j] = make_float2(m_run, l_run);
-      else
-        mass[(int64_t)hk * L_k + j] = (a0 + a1) + (a2 + a3);
-    }
     }
   }
 
@@ -259,7 +299,7 @@ score_mass_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_const
   tc_fence_before();
   __syncthreads();
   if (tid == 0 && *abort && status) atomicOr(status, FC_DEV_TIMEOUT);
-  if (warp == 0) tmem_dealloc(tmem, 2 * kQueries);
+  if (warp == 0) tmem_dealloc(tmem, kRing * kQueries);
 }
 
 }  // namespace
@@ -271,13 +311,13 @@ template <int D, bool kStats>
 int launch(fc_ctx* ctx, cudaStream_t st, const CUtensorMap& t_stream, const CUtensorMap& t_own, int H, int n_stream,
            int n_own, float scale_log2, const float* nlse, float2* ml, int n_slices, float* mass, uint32_t* status) {
   const int n_st = (n_stream + kQueries - 1) / kQueries, n_ot = (n_own + kKeys - 1) / kKeys;
-  // at least 97 KiB, so that a third CTA (and its 256 columns) never joins the SM
-  const size_t need = (1 + kQRing) * (size_t)kKeys * D * 2 + sizeof(MassSmem) + (kStats ? 0 : (size_t)n_st * kQueries * 4) + 1024;
-  const size_t smem = std::max<size_t>(need, 97 * 1024);
-  if (smem > 227 * 1024) return FC_ERR_UNSUPPORTED;  // above 113 KiB one CTA per SM instead of two
-  // two CTAs per SM over all heads; every CTA stays inside one head
-  const int per_sm = smem <= 113 * 1024 ? 2 : 1;
-  dim3 grid(std::max(1, std::min(n_ot, (per_sm * ctx->sm_count) / H)), H, kStats ? n_slices : 1);
+  // at least 120 KiB, so that a second CTA (and its 512 columns) never joins the SM
+  const size_t need = (2 + kRing) * (size_t)kKeys * D * 2 + sizeof(MassSmem) + (kStats ? 0 : (size_t)n_st * kQueries * 4) + 1024;
+  const size_t smem = std::max<size_t>(need, 120 * 1024);
+  if (smem > 227 * 1024) return FC_ERR_UNSUPPORTED;
+  // one CTA per SM over all heads; every CTA stays inside one head.  The statistics launch has few own tiles per
+  // head and slices the streamed range instead (every CTA one own tile).
+  dim3 grid(kStats ? n_ot : std::max(1, std::min(n_ot, ctx->sm_count / H)), H, kStats ? n_slices : 1);
   FC_CUDA_CHECK(cudaFuncSetAttribute(score_mass_kernel<D, kStats>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   score_mass_kernel<D, kStats><<<grid, kThreads, smem, st>>>(t_stream, t_own, n_stream, n_own, scale_log2, nlse, ml, mass,
                                                              status);
@@ -290,13 +330,12 @@ int score_frame_slices(fc_ctx* ctx, int H, int L_q, int L_k) {
   // Slices of the key range in the statistics launch: with few query tiles per head the (head, query tile) pairs
   // alone do not fill the CTA slots evenly.  Cost model: waves of CTAs x (key tiles per slice + 3 tiles' worth of
   // set-up per CTA).
-  const int n_qt = (L_q + kKeys - 1) / kKeys, n_kt = (L_k + kQueries - 1) / kQueries, slots = 2 * ctx->sm_count;
+  const int n_qt = (L_q + kKeys - 1) / kKeys, n_kt = (L_k + kQueries - 1) / kQueries, slots = ctx->sm_count;
   int best = 1;
   int64_t best_cost = INT64_MAX;
   for (int sl = 1; sl <= kScoreFrameMaxSlices && sl <= n_kt; ++sl) {
-    const int64_t ctas = (int64_t)std::min(n_qt, std::max(1, slots / H)) * H * sl;
-    const int64_t own_per_cta = (n_qt + std::max(1, slots / H) - 1) / std::max(1, slots / H);
-    const int64_t cost = ((ctas + slots - 1) / slots) * own_per_cta * ((n_kt + sl - 1) / sl + 3);
+    const int64_t ctas = (int64_t)n_qt * H * sl;
+    const int64_t cost = ((ctas + slots - 1) / slots) * ((n_kt + sl - 1) / sl + 3);
     if (cost < best_cost) {
       best_cost = cost;
       best = sl;

@@ -176,6 +176,75 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
                : "memory");
 }
 
+// Groups of MMAs issued as one block of instructions, every operand already in a register.  The issuing thread
+// does not run ahead of the tensor pipe: what it executes between two MMAs of its own is time during which the
+// pipe has nothing from it (measured: 64 clocks per 128x128x16 MMA back to back, plus 6 to 9 clocks for every
+// instruction in between).  So descriptors are computed, and pinned in registers, before the wait that precedes a group.
+template <int N>
+__device__ __forceinline__ void pin(uint64_t (&d)[N]) {
+  static_assert(N == 4 || N == 8, "group size");
+  if constexpr (N == 8)
+    asm volatile("" : "+l"(d[0]), "+l"(d[1]), "+l"(d[2]), "+l"(d[3]), "+l"(d[4]), "+l"(d[5]), "+l"(d[6]), "+l"(d[7]));
+  else
+    asm volatile("" : "+l"(d[0]), "+l"(d[1]), "+l"(d[2]), "+l"(d[3]));
+}
+__device__ __forceinline__ void pin(uint32_t (&d)[4]) {
+  asm volatile("" : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]));
+}
+// D = A B over N k-steps, A and B in shared memory; the first k-step overwrites D
+template <int N>
+__device__ __forceinline__ void umma_ss_group(uint32_t d_tmem, const uint64_t (&a)[N], const uint64_t (&b)[N], uint32_t idesc) {
+  if constexpr (N == 8) {
+    asm volatile(
+        "{\n"
+        ".reg .pred f, t;\n"
+        "setp.ne.b32 f, %0, %0;\n"
+        "setp.eq.b32 t, %0, %0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %10, %1, f;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %11, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %12, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %5, %13, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %6, %14, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %7, %15, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %8, %16, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %9, %17, %1, t;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(idesc), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]),
+          "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7])
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n"
+        ".reg .pred f, t;\n"
+        "setp.ne.b32 f, %0, %0;\n"
+        "setp.eq.b32 t, %0, %0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %6, %1, f;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %7, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %8, %1, t;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %5, %9, %1, t;\n"
+        "}\n"
+        ::"r"(d_tmem), "r"(idesc), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3])
+        : "memory");
+  }
+}
+// D (+)= A B over 4 k-steps, A in tensor memory; the first k-step accumulates only if `accumulate`
+__device__ __forceinline__ void umma_ts_group(uint32_t d_tmem, const uint32_t (&a)[4], const uint64_t (&b)[4], uint32_t idesc,
+                                              uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p, t;\n"
+      "setp.ne.b32 p, %2, 0;\n"
+      "setp.eq.b32 t, %0, %0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%3], %7, %1, p;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%4], %8, %1, t;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%5], %9, %1, t;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%6], %10, %1, t;\n"
+      "}\n"
+      ::"r"(d_tmem), "r"(idesc), "r"(accumulate), "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "l"(b[0]), "l"(b[1]), "l"(b[2]),
+        "l"(b[3])
+      : "memory");
+}
+
 // ---- two-wide fp32 arithmetic and friends ------------------------------------------------------
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;

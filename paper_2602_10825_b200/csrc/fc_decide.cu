@@ -104,19 +104,37 @@ decide_finalize_kernel(DecideGeom g, const double2* __restrict__ partial,
                        float* __restrict__ l1rel, uint8_t* __restrict__ recompute,
                        int32_t* __restrict__ active_ids, int32_t* __restrict__ n_active) {
   __shared__ uint8_t flag[FC_MAX_CHUNKS];
+  __shared__ double2 part[32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  for (int c = warp; c < g.n_chunks; c += 32) {
+  // The 32 warps are shared out over the chunks, a power of two of them per chunk (all 32 for one chunk, one each
+  // for 32 or more): every warp adds up a fixed subset of the chunk's slabs, the warps of a chunk are combined in
+  // warp order.  Fixed order throughout: bit-reproducible.
+  int wpc = 32;
+  while (wpc > 1 && wpc * min(g.n_chunks, 32) > 32) wpc >>= 1;
+  const int per_round = 32 / wpc;  // chunks handled at a time
+  for (int c0 = 0; c0 < g.n_chunks; c0 += per_round) {
+    const int c = c0 + warp / wpc, sub = warp % wpc;
     double num = 0.0, den = 0.0;
-    for (int s = g.slab_off[c] + lane; s < g.slab_off[c + 1]; s += 32) {
-      num += partial[s].x;
-      den += partial[s].y;
+    if (c < g.n_chunks) {
+      for (int s = g.slab_off[c] + sub * 32 + lane; s < g.slab_off[c + 1]; s += wpc * 32) {
+        num += partial[s].x;
+        den += partial[s].y;
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       num += __shfl_down_sync(0xffffffffu, num, o);
       den += __shfl_down_sync(0xffffffffu, den, o);
     }
-    if (lane == 0) {
+    if (lane == 0) part[warp] = make_double2(num, den);
+    __syncthreads();
+    if (sub == 0 && lane == 0 && c < g.n_chunks) {
+      num = 0.0;
+      den = 0.0;
+      for (int w = 0; w < wpc; ++w) {
+        num += part[warp + w].x;
+        den += part[warp + w].y;
+      }
       double r;
       if (den > 0.0)
         r = num / den;
@@ -130,6 +148,7 @@ decide_finalize_kernel(DecideGeom g, const double2* __restrict__ partial,
       acc[c] = rec ? 0.f : s;
       flag[c] = rec ? 1 : 0;
     }
+    __syncthreads();  // part[] is reused by the next round
   }
   __syncthreads();
   if (threadIdx.x == 0) {

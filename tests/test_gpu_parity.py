@@ -348,6 +348,15 @@ def test_score_frame_level_queries(ctx, d, L_q, L_k):
     _score_case(ctx, Q, K, 0.07, 7)
 
 
+def test_score_frame_level_full_size_two_heads(ctx):
+    # one latent frame of queries (1560 rows) against the 24960 candidates of config 2, two heads (the oracle's
+    # cost grows with the head count; the kernels' work per head does not depend on it)
+    w = wl.CONFIGS["single_step_bf16"]
+    Q = wl.normal((2, 1560, w.d), 81, w.sigma, torch.bfloat16)
+    K = wl.normal((2, w.L_k, w.d), 82, w.sigma, torch.bfloat16)
+    _score_case(ctx, Q, K, w.lam, w.pool_k)
+
+
 def test_score_frame_level_accumulated_over_steps(ctx):
     K = wl.normal((2, 900, 128), 71, 0.5, torch.bfloat16)
     Qs = [wl.normal((2, 200, 128), 72 + s, 0.5, torch.bfloat16) for s in range(2)]

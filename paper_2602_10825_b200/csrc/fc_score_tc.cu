@@ -18,11 +18,12 @@
 //                                   by CUDA cores
 // The finalize step (softmax of a, max-pool, lambda-mix) is the one the CUDA-core path uses.
 //
-// A CTA owns one (head, slice of key tiles).  Warps 0-3 read the logits from tensor memory; warps 4-7 read the
-// key tile from shared memory in pass 1 (norms, column sums) and are a second logit warpgroup in pass 2 (the
-// two take alternate tiles); warp 8 streams key tiles through a
-// 4-stage TMA ring and issues the MMAs into a 2-deep tensor-memory ring.  Keys are read from HBM once: the
-// second pass finds them in L2 for the cache sizes of the paper (a head is a few MB).
+// A CTA owns one (head, slice of key tiles).  Pass 1 (640 threads): two warpgroups read the logits from tensor
+// memory and two read the key tile from shared memory (norms, column sums), each pair taking alternate tiles; one
+// warp streams key tiles through a 4-stage TMA ring and issues the MMAs into a 2-deep tensor-memory ring (one
+// accumulator per logit warpgroup).  Pass 2 (288 threads): no key-vector work, two logit warpgroups on alternate
+// tiles.  Keys are read from HBM once: the second pass finds them in L2 for the cache sizes of the paper (a head is
+// a few MB).
 // Sums are fixed-order: results are bit-reproducible from run to run.  Every mbarrier wait is bounded.
 #include <cmath>
 
@@ -37,15 +38,23 @@ using namespace fc::sm100;
 
 constexpr int kKeys = 128;     // keys per tile
 constexpr int kRing = 4;       // key tiles in flight
-constexpr int kThreads = 288;  // warps 0-3 logits, warps 4-7 key vectors, warp 8 copies and MMAs
+// pass 1: warps 0-3 and 4-7 logits, warps 8-11 and 12-15 key vectors (each pair of warpgroups takes alternate
+//         tiles: one warp per scheduler doing either job alone is bound by the latency of its own instruction
+//         stream), warp 16 copies and MMAs, warps 17-19 idle (whole warpgroups only)
+// pass 2: warps 0-3 and 4-7 logits (alternate tiles), warp 8 copies and MMAs
+template <int PASS>
+constexpr int kThreadsOf = PASS == 1 ? 640 : 288;
+template <int PASS>
+constexpr int kCopyWarp = PASS == 1 ? 16 : 8;
 constexpr int kNQ = fc::kScoreTcMaxQueries;  // queries of pass 2 (MMA N), zero-padded
 
 struct TcSmem {
   uint64_t q_full, q_patched, k_full[kRing], k_free[kRing], s_full[2], s_free[2];
   uint32_t tmem_base, abort;
-  float inv_s[2][kKeys];   // 1 / |k| of the current tile's keys (double-buffered by tile parity)
+  float inv_s[2][kKeys];   // 1 / |k| of the current tile's keys, per key-vector warpgroup (= tile parity)
+  float2 ml_s[kNQ];        // pass 1: (max, sum) of the second logit warpgroup, merged by the first
   alignas(8) float lse_s[kNQ];  // pass 2: minus the log2-domain log-sum-exp per query (-inf for padding queries)
-  float colsum_s[16][128];  // pass 1: per row-group column sums at the end of the slice
+  float colsum_s[2][16][128];  // pass 1: per warpgroup and row group, column sums at the end of the slice
 };
 
 // 16-byte chunk `c` of key row `r` inside a 128-byte-swizzled tile of 64-element column blocks
@@ -55,12 +64,12 @@ __device__ __forceinline__ uint4 lds_key_chunk(const uint8_t* tile, int r, int c
   return *reinterpret_cast<const uint4*>(tile + x * (kKeys * 128) + r * 128 + ((cc ^ (r & 7)) << 4));
 }
 
-__device__ __forceinline__ void named_barrier_128() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void named_barrier_128(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 
 // PASS 1: ml_part [H, n_slices, kNQ] (max, sum) in the log2 domain; colsum_part [H, n_slices, D]
 // PASS 2: imp / a / a_partial as in the CUDA-core path
 template <int D, int PASS>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsOf<PASS>, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                 const fc::ScoreTcArgs g) {
   constexpr uint32_t kTileBytes = kKeys * D * 2;
@@ -122,7 +131,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = sh->tmem_base;
 
-  if (warp == 8) {
+  if (warp == kCopyWarp<PASS>) {
     // ---------------------------------------------------------------- copies and MMAs (one thread)
     if (lane == 0 && n > 0) {
       auto load_k = [&](int i) {  // i-th tile of the CTA into stage i % kRing
@@ -160,59 +169,74 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
       }
     }
-  } else if (warp < 4 || (PASS == 2 && warp < 8)) {
+  } else if (warp < 8) {
     // ---------------------------------------------------------------- logits out of tensor memory
     // (pass 2 has no key-vector work, so warps 4-7 are a second logit warpgroup: the two take alternate tiles,
     // each the tensor-memory buffer of its own parity)
     const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     if (PASS == 1) {
-      const int q = tid;  // query row
+      const int grp = warp >> 2;  // this warpgroup takes the tiles of its parity and the accumulator of that parity
+      const int q = tid & 127;    // query row
       const bool row_ok = q < g.L_q;
-      const bool warp_ok = warp * 32 < g.L_q;
+      const bool warp_ok = (warp & 3) * 32 < g.L_q;
       float m = -INFINITY, l = 0.f;
-      for (int i = 0; i < n; ++i) {
-        const int b = i & 1;
+      for (int i = grp; i < n; i += 2) {
+        const int b = grp;
         mbar_wait_bounded(smem_u32(&sh->s_full[b]), (i >> 1) & 1, abort);
         tc_fence_after();
-        uint32_t sv[kKeys];
-        if (warp_ok) tmem_ld128_wait(t_lane + b * kCols, sv);
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
-        if (!warp_ok) continue;
         const int cols_valid = min(kKeys, g.L_k - tile_of(i) * kKeys);
-        if (cols_valid < kKeys) {
+        // 64 columns at a time (a 128-column row per thread does not fit the registers of a 640-thread CTA)
 #pragma unroll
-          for (int c = 0; c < kKeys; ++c)
-            if (c >= cols_valid) sv[c] = 0xff800000u;  // -inf
-        }
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        for (int half = 0; half < 2; ++half) {
+          uint32_t sv[64];
+          if (warp_ok) tmem_ld64_wait(t_lane + b * kCols + half * 64, sv);
+          if (half == 1) {  // the accumulator can take this warpgroup's next tile
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->s_free[b]));
+          }
+          if (!warp_ok) continue;
+          if (cols_valid < half * 64 + 64) {
 #pragma unroll
-        for (int c = 0; c < kKeys; c += 8) {
+            for (int c = 0; c < 64; ++c)
+              if (half * 64 + c >= cols_valid) sv[c] = 0xff800000u;  // -inf
+          }
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (int c4 = 0; c4 < 4; ++c4)
-            mx[c4] = max3(mx[c4], __uint_as_float(sv[c + 2 * c4]), __uint_as_float(sv[c + 2 * c4 + 1]));
-        }
-        const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * g.scale_log2;  // scale > 0
-        if (tile_max > m) {
-          l *= ex2(m - tile_max);  // 0 on the first tile
-          m = tile_max;
-        }
-        const uint64_t sc2 = pack2(g.scale_log2, g.scale_log2), nm2 = pack2(-m, -m);
-        uint64_t sum2[2] = {0ull, 0ull};
+          for (int c = 0; c < 64; c += 8) {
 #pragma unroll
-        for (int c = 0; c < kKeys; c += 2) {
-          const uint64_t x = fma2(pack2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), sc2, nm2);
-          float x0, x1;
-          unpack2(x, x0, x1);
-          sum2[(c >> 1) & 1] = add2(sum2[(c >> 1) & 1], pack2(ex2(x0), ex2(x1)));
+            for (int c4 = 0; c4 < 4; ++c4)
+              mx[c4] = max3(mx[c4], __uint_as_float(sv[c + 2 * c4]), __uint_as_float(sv[c + 2 * c4 + 1]));
+          }
+          const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * g.scale_log2;  // scale > 0
+          if (tile_max > m) {
+            l *= ex2(m - tile_max);  // 0 on the first tile
+            m = tile_max;
+          }
+          const uint64_t sc2 = pack2(g.scale_log2, g.scale_log2), nm2 = pack2(-m, -m);
+          uint64_t sum2[2] = {0ull, 0ull};
+#pragma unroll
+          for (int c = 0; c < 64; c += 2) {
+            const uint64_t x = fma2(pack2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), sc2, nm2);
+            float x0, x1;
+            unpack2(x, x0, x1);
+            sum2[(c >> 1) & 1] = add2(sum2[(c >> 1) & 1], pack2(ex2(x0), ex2(x1)));
+          }
+          float a0, a1, a2, a3;
+          unpack2(sum2[0], a0, a1);
+          unpack2(sum2[1], a2, a3);
+          l += (a0 + a1) + (a2 + a3);
         }
-        float a0, a1, a2, a3;
-        unpack2(sum2[0], a0, a1);
-        unpack2(sum2[1], a2, a3);
-        l += (a0 + a1) + (a2 + a3);
       }
-      if (row_ok) g.ml_part[((int64_t)hk * g.n_slices + slice) * kNQ + q] = make_float2(m, l);
+      // the two warpgroups' results of the slice, merged in group order
+      if (grp == 1 && q < kNQ) sh->ml_s[q] = make_float2(m, l);
+      asm volatile("bar.sync 4, 256;" ::: "memory");
+      if (grp == 0 && row_ok) {
+        const float2 p = sh->ml_s[q];
+        const float mn = fmaxf(m, p.x);
+        const float lm = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * exp2f(p.x - mn));
+        g.ml_part[((int64_t)hk * g.n_slices + slice) * kNQ + q] = make_float2(mn, lm);
+      }
     } else {
       // The mean key joins the queries as rows kNQ-2 (bf16 high part) and kNQ-1 (low part) of the Q tile, which
       // the copy zero-filled: generic-proxy writes, made visible to the tensor cores by the proxy fence.
@@ -291,9 +315,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         if (lane == 0) g.a_partial[((int64_t)hk * g.n_tiles + tile_id) * 4 + (warp & 3)] = make_float2(m, l);
       }
     }
-  } else if (PASS == 1) {
+  } else if (PASS == 1 && warp < 16) {
     // ---------------------------------------------------------------- key vectors out of shared memory
-    const int u = tid - 128;  // 0..127
+    const int vg = (tid - 256) >> 7;  // warpgroup 0 or 1: the tiles of its parity
+    const int u = (tid - 256) & 127;  // 0..127
     {
       // column sums of the normalised keys: this thread owns 16-byte chunk `c` of the rows r = rg (mod kGroups)
       constexpr int kGroups = 128 / kChunks;  // 8 for d = 128, 16 for d = 64
@@ -301,7 +326,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       float acc[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-      for (int i = 0; i < n; ++i) {
+      for (int i = vg; i < n; i += 2) {
         const int st = i % kRing;
         mbar_wait_bounded(smem_u32(&sh->k_full[st]), (i / kRing) & 1, abort);
         const uint8_t* tile = k_tiles + st * kTileBytes;
@@ -321,11 +346,11 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         const int j = tile_of(i) * kKeys + u;
         if (j < g.L_k) g.norm2[(int64_t)hk * g.L_k + j] = n2;  // pass 2 takes |k|^2 from here
         // rows past the end of the cache are zero-filled: 0 * (1 / 1e-12) = 0, they add nothing
-        sh->inv_s[i & 1][u] = 1.f / fmaxf(sqrtf(n2), 1e-12f);
-        named_barrier_128();
+        sh->inv_s[vg][u] = 1.f / fmaxf(sqrtf(n2), 1e-12f);
+        named_barrier_128(1 + vg);
         for (int r = rg; r < kKeys; r += kGroups) {
           const uint4 w = lds_key_chunk<D>(tile, r, c);
-          const float inv = sh->inv_s[i & 1][r];
+          const float inv = sh->inv_s[vg][r];
           const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -333,15 +358,17 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
             acc[2 * e + 1] = fmaf(fc::bf16_hi(ww[e]), inv, acc[2 * e + 1]);
           }
         }
+        named_barrier_128(1 + vg);  // inv_s[vg] is rewritten for this warpgroup's next tile
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sh->k_free[st]));
       }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) sh->colsum_s[rg][c * 8 + e] = acc[e];
-      named_barrier_128();
-      if (u < D) {
+      for (int e = 0; e < 8; ++e) sh->colsum_s[vg][rg][c * 8 + e] = acc[e];
+      asm volatile("bar.sync 3, 256;" ::: "memory");  // both key-vector warpgroups
+      if (vg == 0 && u < D) {
         float t = 0.f;
-        for (int r = 0; r < kGroups; ++r) t += sh->colsum_s[r][u];
+        for (int v = 0; v < 2; ++v)
+          for (int r = 0; r < kGroups; ++r) t += sh->colsum_s[v][r][u];
         g.colsum_part[((int64_t)hk * g.n_slices + slice) * D + u] = t;
       }
     }
@@ -373,14 +400,15 @@ int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs g, int d, int64_t q_h
   g.n_slices = (g.n_tiles + g.tiles_per_slice - 1) / g.tiles_per_slice;  // no empty slice
   const size_t smem = (size_t)(1 + kRing) * kKeys * d * 2 + sizeof(TcSmem) + 1024;
   const dim3 grid(g.n_slices, g.H);
-  auto launch = [&](auto kernel) -> int {
+  auto launch = [&](auto kernel, int threads) -> int {
     FC_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kernel<<<grid, kThreads, smem, st>>>(tq, tk, g);
+    kernel<<<grid, threads, smem, st>>>(tq, tk, g);
     FC_LAUNCH_CHECK("score_tc_kernel");
     return FC_OK;
   };
-  if ((rc = d == 128 ? launch(score_tc_kernel<128, 1>) : launch(score_tc_kernel<64, 1>)) != FC_OK) return rc;
-  return d == 128 ? launch(score_tc_kernel<128, 2>) : launch(score_tc_kernel<64, 2>);
+  if ((rc = d == 128 ? launch(score_tc_kernel<128, 1>, kThreadsOf<1>) : launch(score_tc_kernel<64, 1>, kThreadsOf<1>)) != FC_OK)
+    return rc;
+  return d == 128 ? launch(score_tc_kernel<128, 2>, kThreadsOf<2>) : launch(score_tc_kernel<64, 2>, kThreadsOf<2>);
 }
 
 }  // namespace fc

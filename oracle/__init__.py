@@ -107,6 +107,45 @@ def chunk_decide(cur, prev, chunk_elem_off, chunk_step, warmup_m, eps, acc,
                 n_active=int(cnt[0]))
 
 
+def chunk_decide_uniform(cur, prev, chunk_elem_off, chunk_step, warmup_m, eps, acc,
+                         force=None, n_threads=0):
+    """The uniform policy of the caption of Fig. 3 (one shared decision; forced and warm-up chunks
+    are computed anyway).  Same returns as chunk_decide."""
+    off = np.ascontiguousarray(np.asarray(chunk_elem_off, dtype=np.int64))
+    n = len(off) - 1
+    step = _i32(chunk_step)
+    acc_out = np.array(acc, dtype=np.float32, copy=True)
+    l1rel = np.zeros(n, np.float32)
+    rec = np.zeros(n, np.uint8)
+    ids = np.full(n, -1, np.int32)
+    cnt = np.zeros(1, np.int32)
+    frc = None if force is None else np.ascontiguousarray(np.asarray(force, dtype=np.uint8))
+    rc = lib().fco_chunk_decide_uniform(_ptr(cur), _ptr(prev), _dtype_of(cur), _ptr(off), n,
+                                        _ptr(step), int(warmup_m), C.c_float(eps), _ptr(frc),
+                                        _ptr(acc_out), _ptr(l1rel), _ptr(rec), _ptr(ids),
+                                        _ptr(cnt), int(n_threads))
+    if rc:
+        raise ValueError(f"fco_chunk_decide_uniform -> {rc}")
+    return dict(l1rel=l1rel, recompute=rec, acc=acc_out, active_ids=ids[:cnt[0]].copy(),
+                n_active=int(cnt[0]))
+
+
+def chunk_cache_apply(x_in, y, cache, chunk_elem_off, recompute, n_threads=0):
+    """Activation-cache step (Sec. 3.2): computed chunks store y - x into the cache, skipped chunks
+    get y = x + cache.  Returns new (y, cache) arrays; the inputs are not modified."""
+    off = np.ascontiguousarray(np.asarray(chunk_elem_off, dtype=np.int64))
+    n = len(off) - 1
+    y_out = np.array(y, copy=True)
+    c_out = np.array(cache, copy=True)
+    rec = np.ascontiguousarray(np.asarray(recompute, dtype=np.uint8))
+    assert x_in.dtype == y_out.dtype == c_out.dtype and len(rec) == n
+    rc = lib().fco_chunk_cache_apply(_ptr(np.ascontiguousarray(x_in)), _ptr(y_out), _ptr(c_out),
+                                     _dtype_of(y_out), _ptr(off), n, _ptr(rec), int(n_threads))
+    if rc:
+        raise ValueError(f"fco_chunk_cache_apply -> {rc}")
+    return y_out, c_out
+
+
 def chunk_attention(Q, K, V, q_chunk_row_off, kv_visible_len, seg_logical_off,
                     seg_phys_off, active_ids, *, H_kv=None, scale=0.0,
                     kv_token_index=None, sample_rows=None, O_init=None, n_threads=0):

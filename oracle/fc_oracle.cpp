@@ -107,6 +107,126 @@ extern "C" int fco_chunk_decide(const void* cur, const void* prev, int dtype,
 }
 
 // ---------------------------------------------------------------------------
+// The uniform ("traditional reuse") policy of the caption of Fig. 3: all chunks
+// of a timestep share ONE compute / reuse status, except chunks that must be
+// computed anyway (newly initialised: still in warm-up, or forced).  The shared
+// indicator is Eq. 4 taken over all sharing chunks as one tensor; the shared
+// accumulator follows Eq. 8.
+// ---------------------------------------------------------------------------
+extern "C" int fco_chunk_decide_uniform(const void* cur, const void* prev, int dtype,
+                                        const int64_t* chunk_elem_off, int n_chunks,
+                                        const int32_t* chunk_step, int warmup_m,
+                                        float eps, const uint8_t* force, float* acc,
+                                        float* l1rel, uint8_t* recompute,
+                                        int32_t* active_ids, int32_t* n_active,
+                                        int n_threads) {
+  if (!chunk_elem_off || !chunk_step || !acc || !recompute || n_chunks < 0)
+    return -1;
+  if (dtype != FCO_BF16 && dtype != FCO_F32) return -2;
+  std::vector<double> num(n_chunks, 0.0), den(n_chunks, 0.0);
+  parallel_for(n_chunks, n_threads, [&](int64_t c) {
+    for (int64_t e = chunk_elem_off[c]; e < chunk_elem_off[c + 1]; ++e) {
+      double x_prev = widen(prev, dtype, e), x_cur = widen(cur, dtype, e);
+      num[c] += std::fabs(x_cur - x_prev);
+      den[c] += std::fabs(x_prev);
+    }
+  });
+  auto ratio = [](double n, double d) {
+    if (d > 0.0) return n / d;
+    return n > 0.0 ? std::numeric_limits<double>::infinity() : 0.0;
+  };
+  // the chunks that share the decision, and their common indicator
+  double num_all = 0.0, den_all = 0.0;
+  int first_sharing = -1;
+  std::vector<uint8_t> own(n_chunks, 0);
+  for (int c = 0; c < n_chunks; ++c) {
+    own[c] = (chunk_step[c] < warmup_m) || (force && force[c]);
+    if (own[c]) continue;
+    if (first_sharing < 0) first_sharing = c;
+    num_all += num[c];
+    den_all += den[c];
+  }
+  bool shared_compute = true;
+  float acc_next = 0.0f;
+  float r_shared = 0.0f;
+  if (first_sharing >= 0) {
+    r_shared = (float)ratio(num_all, den_all);
+    volatile float s = acc[first_sharing] + r_shared;  // fp32, as in Eq. 8's accumulator
+    shared_compute = s > eps;
+    acc_next = shared_compute ? 0.0f : s;
+  }
+  int32_t count = 0;
+  for (int c = 0; c < n_chunks; ++c) {
+    if (l1rel) l1rel[c] = own[c] ? (float)ratio(num[c], den[c]) : r_shared;
+    recompute[c] = (own[c] || shared_compute) ? 1 : 0;
+    acc[c] = acc_next;
+    if (recompute[c]) {
+      if (active_ids) active_ids[count] = c;
+      ++count;
+    }
+  }
+  if (n_active) *n_active = count;
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Sec. 3.2 (text after Eq. 8): a chunk that is not recomputed is served from
+// its cached activations.  The cache holds, per chunk, the residual between the
+// output and the input of the last computed forward; a reused chunk's output is
+// its current input plus that residual.  Arithmetic is in fp32 and rounded once
+// to the storage type (the result is a stored code: both sides of a parity test
+// must round the same fp32 value).
+// ---------------------------------------------------------------------------
+namespace {
+inline float load_f32(const void* base, int dtype, int64_t i) {
+  if (dtype == FCO_F32) return static_cast<const float*>(base)[i];
+  uint32_t bits = (uint32_t)static_cast<const uint16_t*>(base)[i] << 16;
+  float f;
+  std::memcpy(&f, &bits, sizeof f);
+  return f;
+}
+inline void store_rounded(void* base, int dtype, int64_t i, float v) {
+  if (dtype == FCO_F32) {
+    static_cast<float*>(base)[i] = v;
+    return;
+  }
+  uint32_t u;
+  std::memcpy(&u, &v, sizeof u);
+  uint16_t out;
+  if ((u & 0x7fffffffu) > 0x7f800000u) {
+    out = (uint16_t)((u >> 16) | 0x0040u);  // NaN stays NaN (quiet)
+  } else {
+    // round to nearest, ties to even, on the 16 bits that are dropped
+    uint32_t lsb = (u >> 16) & 1u;
+    out = (uint16_t)((u + 0x7fffu + lsb) >> 16);
+  }
+  static_cast<uint16_t*>(base)[i] = out;
+}
+}  // namespace
+
+extern "C" int fco_chunk_cache_apply(const void* x_in, void* y_io, void* cache, int dtype,
+                                     const int64_t* chunk_elem_off, int n_chunks,
+                                     const uint8_t* recompute, int n_threads) {
+  if (!chunk_elem_off || !recompute || n_chunks < 0) return -1;
+  if (dtype != FCO_BF16 && dtype != FCO_F32) return -2;
+  parallel_for(n_chunks, n_threads, [&](int64_t c) {
+    for (int64_t e = chunk_elem_off[c]; e < chunk_elem_off[c + 1]; ++e) {
+      const float x = load_f32(x_in, dtype, e);
+      if (recompute[c]) {
+        // the forward ran: remember what it added to its input
+        volatile float delta = load_f32(y_io, dtype, e) - x;
+        store_rounded(cache, dtype, e, delta);
+      } else {
+        // the forward was skipped: input plus the remembered residual
+        volatile float y = x + load_f32(cache, dtype, e);
+        store_rounded(y_io, dtype, e, y);
+      }
+    }
+  });
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
 // Sec. 3.3: queries of the chunks being denoised attend to the compressed
 // clean-chunk region followed by the denoising region; chunk c sees a logical
 // prefix of kv_visible_len[c] tokens.  Textbook softmax attention per row.

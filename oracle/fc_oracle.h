@@ -40,6 +40,31 @@ int fco_chunk_decide(const void* cur, const void* prev, int dtype,
                      uint8_t* recompute, int32_t* active_ids,
                      int32_t* n_active, int n_threads);
 
+/* The uniform ("traditional reuse") policy the paper compares with (caption of
+ * Fig. 3): every chunk of a timestep shares one compute / reuse status, except
+ * chunks that must be computed anyway (chunk_step[i] < warmup_m, or force[i]).
+ * Over the sharing chunks S taken as one tensor:
+ *   r = sum_S |cur - prev| / sum_S |prev|  (fp64, rounded to fp32);
+ *   s = acc[first chunk of S] + r in fp32; all of S is recomputed iff s > eps;
+ *   every acc[i] <- 0 if so, else s (all entries stay equal; 0 if S is empty).
+ * l1rel[i] = r for i in S, the chunk's own indicator otherwise. */
+int fco_chunk_decide_uniform(const void* cur, const void* prev, int dtype,
+                             const int64_t* chunk_elem_off, int n_chunks,
+                             const int32_t* chunk_step, int warmup_m, float eps,
+                             const uint8_t* force, float* acc, float* l1rel,
+                             uint8_t* recompute, int32_t* active_ids,
+                             int32_t* n_active, int n_threads);
+
+/* Serving skipped chunks from the activation cache (Sec. 3.2, text after Eq. 8).
+ * For every element e of chunk i (same flat layout as fco_chunk_decide):
+ *   recompute[i] != 0:  cache[e] <- round(y[e] - x[e])      (y: the fresh output)
+ *   recompute[i] == 0:  y[e]     <- round(x[e] + cache[e])  (cache is not modified)
+ * with the difference / sum taken in fp32 and rounded once to the storage type
+ * (round to nearest even for bf16). */
+int fco_chunk_cache_apply(const void* x_in, void* y_io, void* cache, int dtype,
+                          const int64_t* chunk_elem_off, int n_chunks,
+                          const uint8_t* recompute, int n_threads);
+
 typedef struct {
   int32_t H_q, H_kv, d, W;
   int64_t q_hs, q_rs, k_hs, k_rs, v_hs, v_rs; /* element strides: head, row */

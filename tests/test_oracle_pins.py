@@ -384,3 +384,101 @@ def test_attention_on_compacted_cache_equals_token_map_on_uncompacted():
                                       kv_token_index=tok)
     assert np.array_equal(O_compact, O_map)
     assert L_phys == 14
+
+
+# --------------------------------------------------------------------------- uniform policy (caption of Fig. 3)
+
+def test_uniform_policy_hand_trace(golden):
+    g = golden("uniform_policy_hand_trace.txt")
+    eps, m, n_el = g["eps"][0], int(g["warmup_m"][0]), 4096
+    acc = np.zeros(3, np.float32)
+    for s in range(len(g["acc_after"])):
+        target = [g["r_chunk0"][s], g["r_chunk1"][s], g["r_chunk2"][s]]
+        # |prev| = 1 everywhere (random signs), cur = prev (1 +- r): equal weights, so the indicator over several
+        # chunks taken as one tensor is the mean of the chunks' own indicators
+        prev = torch.sign(wl.normal((3 * n_el,), 40 + s)) + 0.0
+        prev[prev == 0] = 1.0
+        alt = torch.where(torch.arange(3 * n_el) % 2 == 0, 1.0, -1.0)
+        cur = prev * (1 + torch.tensor(target, dtype=torch.float32).repeat_interleave(n_el) * alt)
+        step = np.array([s, s, int(g["step_chunk2"][s])], np.int32)
+        out = oracle.chunk_decide_uniform(wl.bits(cur.float()), wl.bits(prev.float()), [0, n_el, 2 * n_el, 3 * n_el],
+                                          step, m, eps, acc)
+        want = [int(g[f"recompute{c}"][s]) for c in range(3)]
+        assert out["recompute"].tolist() == want, f"step {s}"
+        assert out["active_ids"].tolist() == [c for c in range(3) if want[c]]
+        np.testing.assert_allclose(out["acc"], [g["acc_after"][s]] * 3, atol=2e-6)
+        acc = out["acc"]
+
+
+def test_uniform_policy_reduces_to_the_chunkwise_rule_for_one_chunk_and_differs_for_several():
+    # one chunk: the shared decision IS the chunk's decision (Eq. 8)
+    acc_u = acc_c = np.zeros(1, np.float32)
+    for s, r in enumerate([0.08, 0.05, 0.04, 0.09, 0.20, 0.01, 0.13, 0.02]):
+        cur, prev = wl.indicator_pair(1, 2048, [r], 70 + s, dtype=torch.float32)
+        u = oracle.chunk_decide_uniform(wl.bits(cur), wl.bits(prev), [0, 2048], [s], 1, 0.15, acc_u)
+        c = oracle.chunk_decide(wl.bits(cur), wl.bits(prev), [0, 2048], [s], 1, 0.15, acc_c)
+        assert u["recompute"].tolist() == c["recompute"].tolist()
+        np.testing.assert_array_equal(u["acc"], c["acc"])
+        np.testing.assert_array_equal(u["l1rel"], c["l1rel"])
+        acc_u, acc_c = u["acc"], c["acc"]
+    # several chunks: one flag for all sharing chunks, whatever their own indicators; a forced chunk computes anyway
+    # and its elements do not enter the shared indicator
+    n = 1000
+    prev = np.ones(3 * n, np.float32)
+    cur = prev.copy()
+    cur[:n] *= 1.5       # chunk 0 changed by 0.5
+    cur[2 * n:] *= 3.0   # chunk 2 changed by 2.0 but is forced: excluded from the shared sum
+    out = oracle.chunk_decide_uniform(cur, prev, [0, n, 2 * n, 3 * n], [5, 5, 5], 1, 0.3, np.zeros(3, np.float32),
+                                      force=[0, 0, 1])
+    assert out["l1rel"].tolist() == [0.25, 0.25, 2.0]   # (0.5 n + 0) / 2n for the sharing chunks
+    assert out["recompute"].tolist() == [0, 0, 1]        # 0.25 <= 0.3: the sharing chunks reuse
+    np.testing.assert_array_equal(out["acc"], np.float32([0.25, 0.25, 0.25]))
+    out = oracle.chunk_decide_uniform(cur, prev, [0, n, 2 * n, 3 * n], [5, 5, 5], 1, 0.2, np.zeros(3, np.float32),
+                                      force=[0, 0, 1])
+    assert out["recompute"].tolist() == [1, 1, 1] and out["acc"].tolist() == [0.0, 0.0, 0.0]
+    # the shared indicator is the ratio of the sums, not the mean of the ratios: chunks of different magnitude
+    prev2 = np.concatenate([np.ones(n, np.float32), np.full(n, 9.0, np.float32)])
+    cur2 = np.concatenate([np.full(n, 2.0, np.float32), np.full(n, 9.0, np.float32)])  # r0 = 1, r1 = 0
+    out = oracle.chunk_decide_uniform(cur2, prev2, [0, n, 2 * n], [5, 5], 1, 10.0, np.zeros(2, np.float32))
+    assert out["l1rel"].tolist() == [np.float32(0.1)] * 2  # n / (n + 9 n), not (1 + 0) / 2
+    # every chunk forced or warming up: all compute, accumulator cleared
+    out = oracle.chunk_decide_uniform(cur2, prev2, [0, n, 2 * n], [0, 9], 1, 10.0, np.float32([0.3, 0.3]), force=[0, 1])
+    assert out["recompute"].tolist() == [1, 1] and out["acc"].tolist() == [0.0, 0.0]
+
+
+# --------------------------------------------------------------------------- activation cache (Sec. 3.2)
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_cache_apply_hand_example(golden, dtype):
+    g = golden("cache_apply_hand_example.txt")
+    t = lambda k: wl.bits(torch.tensor(g[k], dtype=torch.float32).to(dtype))
+    back = lambda a: (torch.from_numpy(a.copy()).view(torch.bfloat16) if a.dtype == np.uint16 else torch.from_numpy(a)).float().tolist()
+    off = [0, 3, 6]
+    y, cache = oracle.chunk_cache_apply(t("xA"), t("yA"), wl.bits(torch.full((6,), 77.0).to(dtype)), off, [1, 1])
+    assert back(cache) == g["cacheA"] and back(y) == g["yA"]        # computed chunks: y untouched, cache = y - x
+    y, cache = oracle.chunk_cache_apply(t("xB"), t("yB_in"), cache, off, [int(v) for v in g["recB"]])
+    assert back(y) == g["yB_out"] and back(cache) == g["cacheB"]
+
+
+def test_cache_apply_matches_library_arithmetic_and_rounding():
+    # fp32 add / subtract by numpy, rounding to bf16 by torch (round to nearest even): library routines
+    n = 5000
+    x, yv, c = (wl.normal((2 * n,), 300 + i, 3.0, torch.bfloat16) for i in range(3))
+    y, cache = oracle.chunk_cache_apply(wl.bits(x), wl.bits(yv), wl.bits(c), [0, n, 2 * n], [0, 1])
+    want_y = (x.float()[:n] + c.float()[:n]).to(torch.bfloat16)
+    want_c = (yv.float()[n:] - x.float()[n:]).to(torch.bfloat16)
+    assert np.array_equal(y[:n], wl.bits(want_y)) and np.array_equal(y[n:], wl.bits(yv)[n:])
+    assert np.array_equal(cache[n:], wl.bits(want_c)) and np.array_equal(cache[:n], wl.bits(c)[:n])
+    # ties round to even: 1 + 2^-8 is halfway between two bf16 values around 1 -> 1.0; 1 + 3 * 2^-8 -> 1 + 2^-6
+    xs = torch.tensor([1.0, 1.0], dtype=torch.bfloat16)
+    cs = torch.tensor([2.0 ** -8, 3 * 2.0 ** -8], dtype=torch.bfloat16)
+    y, _ = oracle.chunk_cache_apply(wl.bits(xs), wl.bits(xs), wl.bits(cs), [0, 2], [0])
+    assert torch.from_numpy(y.copy()).view(torch.bfloat16).float().tolist() == [1.0, 1.0 + 2.0 ** -6]
+    # fp32 storage: plain fp32 arithmetic, bit for bit
+    xf, yf, cf = (wl.normal((n,), 310 + i, 2.0) for i in range(3))
+    y, cache = oracle.chunk_cache_apply(xf.numpy(), yf.numpy(), cf.numpy(), [0, n // 2, n], [1, 0])
+    assert np.array_equal(cache[:n // 2], (yf - xf).numpy()[:n // 2])
+    assert np.array_equal(y[n // 2:], (xf + cf).numpy()[n // 2:])
+    # a zero residual serves the input back unchanged; an empty chunk is fine
+    y, _ = oracle.chunk_cache_apply(xf.numpy(), yf.numpy(), np.zeros(n, np.float32), [0, 0, n], [0, 0])
+    assert np.array_equal(y, xf.numpy())

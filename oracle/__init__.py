@@ -20,7 +20,7 @@ _SO = os.path.join(_HERE, "libfc_oracle.so")
 _SRC = os.path.join(_HERE, "fc_oracle.cpp")
 
 BF16, F32 = 0, 1
-RED_AUTO, RED_PLAIN, RED_MEANKEY = 0, 1, 2
+RED_AUTO, RED_PLAIN, RED_MEANKEY, RED_MAXSIM = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -202,6 +202,20 @@ def kv_score(Q_obs, K_cand, *, lambda_=0.07, pool_k=7, red_mode=RED_AUTO, scale=
     if rc:
         raise ValueError(f"fco_kv_score -> {rc}")
     return dict(imp=imp, imp_pooled=pooled, red=red, score=score)
+
+
+def key_similarity_columns(K_cand, cols, red_mode=RED_PLAIN, n_threads=0):
+    """The softmax argument of Eq. 11 (column mean of the cosine matrix with zeroed diagonal; or, with
+    RED_MAXSIM, the largest similarity to another token) for the columns ``cols`` only.  [H, len(cols)]."""
+    H, L_k, d = K_cand.shape
+    cols = _i32(cols)
+    out = np.zeros((H, len(cols)), np.float64)
+    rc = lib().fco_key_similarity_columns(_ptr(K_cand), _dtype_of(K_cand), H, L_k, d, C.c_int64(L_k * d),
+                                          C.c_int64(d), _ptr(cols), len(cols), int(red_mode), _ptr(out),
+                                          int(n_threads))
+    if rc:
+        raise ValueError(f"fco_key_similarity_columns -> {rc}")
+    return out
 
 
 def kv_select_compact(score, B, K_src=None, V_src=None, n_threads=0):

@@ -413,7 +413,21 @@ extern "C" int fco_kv_score(const fco_score_desc* desc, const void* Q_obs,
       for (int e = 0; e < d; ++e) khat[(size_t)j * d + e] *= inv;
     }
     std::vector<double> col_mean(L_k, 0.0);
-    if (red_mode == FCO_RED_PLAIN) {
+    if (red_mode == FCO_RED_MAXSIM) {
+      // Variant outside the paper (it does not collapse to a mean key): the similarity of token j to its most
+      // similar OTHER token takes the place of the column mean; the diagonal is excluded, not zeroed.
+      for (int j = 0; j < L_k; ++j) {
+        double best = L_k > 1 ? -std::numeric_limits<double>::infinity() : 0.0;
+        for (int i = 0; i < L_k; ++i) {
+          if (i == j) continue;
+          double dot = 0.0;
+          for (int e = 0; e < d; ++e)
+            dot += khat[(size_t)i * d + e] * khat[(size_t)j * d + e];
+          best = std::max(best, dot);
+        }
+        col_mean[j] = best;
+      }
+    } else if (red_mode == FCO_RED_PLAIN) {
       for (int j = 0; j < L_k; ++j) {
         double acc = 0.0;
         for (int i = 0; i < L_k; ++i) {
@@ -457,6 +471,49 @@ extern "C" int fco_kv_score(const fco_score_desc* desc, const void* Q_obs,
       if (red) red[hk * L_k + j] = red_h[j];
       score[hk * L_k + j] = (float)(lambda * pooled[j] - (1.0 - lambda) * red_h[j]);
     }
+  });
+  return 0;
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 11 before its softmax, for chosen columns only: the column statistic of the
+// cosine-similarity matrix by its plain definition (every other token visited),
+// so that large caches can be checked on a sample of columns.
+// ---------------------------------------------------------------------------
+extern "C" int fco_key_similarity_columns(const void* K_cand, int dtype, int n_heads,
+                                          int L_k, int d, int64_t k_hs, int64_t k_rs,
+                                          const int32_t* cols, int n_cols, int red_mode,
+                                          double* out, int n_threads) {
+  if (!K_cand || !cols || !out || n_heads <= 0 || L_k <= 0 || d <= 0 || n_cols < 0) return -1;
+  if (dtype != FCO_BF16 && dtype != FCO_F32) return -2;
+  if (red_mode != FCO_RED_PLAIN && red_mode != FCO_RED_MAXSIM) return -3;
+  for (int c = 0; c < n_cols; ++c)
+    if (cols[c] < 0 || cols[c] >= L_k) return -4;
+  parallel_for((int64_t)n_heads * n_cols, n_threads, [&](int64_t item) {
+    const int64_t h = item / n_cols;
+    const int j = cols[item % n_cols];
+    auto unit_key = [&](int t, std::vector<double>& v) {
+      double nrm2 = 0.0;
+      for (int e = 0; e < d; ++e) {
+        v[e] = widen(K_cand, dtype, h * k_hs + (int64_t)t * k_rs + e);
+        nrm2 += v[e] * v[e];
+      }
+      const double inv = 1.0 / std::max(std::sqrt(nrm2), 1e-12);
+      for (int e = 0; e < d; ++e) v[e] *= inv;
+    };
+    std::vector<double> kj(d), ki(d);
+    unit_key(j, kj);
+    double sum = 0.0;
+    double best = L_k > 1 ? -std::numeric_limits<double>::infinity() : 0.0;
+    for (int i = 0; i < L_k; ++i) {
+      if (i == j) continue;  // S_jj = 0 (sum) / excluded (max)
+      unit_key(i, ki);
+      double dot = 0.0;
+      for (int e = 0; e < d; ++e) dot += ki[e] * kj[e];
+      sum += dot;
+      best = std::max(best, dot);
+    }
+    out[item] = red_mode == FCO_RED_PLAIN ? sum / (double)L_k : best;
   });
   return 0;
 }

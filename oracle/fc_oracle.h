@@ -24,7 +24,7 @@ extern "C" {
 #endif
 
 enum { FCO_BF16 = 0, FCO_F32 = 1 };
-enum { FCO_RED_AUTO = 0, FCO_RED_PLAIN = 1, FCO_RED_MEANKEY = 2 };
+enum { FCO_RED_AUTO = 0, FCO_RED_PLAIN = 1, FCO_RED_MEANKEY = 2, FCO_RED_MAXSIM = 3 };
 
 /* Per-chunk reuse decision: relative-L1 indicator (Eq. 5, the per-chunk form
  * of Eq. 4) fed to the accumulate / threshold / reset rule (Eq. 8).
@@ -113,6 +113,8 @@ typedef struct {
  * red_mode PLAIN builds the L_k x L_k cosine matrix, zeroes its diagonal and
  * takes column means; MEANKEY uses the appendix identity
  * (mean_i khat_i) . khat_j - |khat_j|^2 / L_k; AUTO = PLAIN up to 4096 tokens.
+ * MAXSIM is a variant outside the paper that no mean key can express: the
+ * softmax argument of token j is max_{i != j} khat_i . khat_j (0 if L_k = 1).
  * accum_phase: 0 single shot; 1 imp_accum += Imp, no outputs; 2 imp_accum +=
  * Imp, Imp := imp_accum / n_steps, then finalise.  Outputs other than score may
  * be NULL. */
@@ -120,6 +122,24 @@ int fco_kv_score(const fco_score_desc* desc, const void* Q_obs,
                  const void* K_cand, int dtype, double* imp_accum,
                  int accum_phase, int n_steps, double* imp, double* imp_pooled,
                  double* red, float* score, int n_threads);
+
+/* The softmax argument of Eq. 11 for chosen columns only, by its plain
+ * definition: out[h][c] = (1/L_k) sum_{i != j} khat_i . khat_j for j = cols[c]
+ * (red_mode PLAIN) or max_{i != j} khat_i . khat_j (MAXSIM).  K_cand is
+ * [n_heads, L_k, d] with strides k_hs, k_rs; out is [n_heads, n_cols]. */
+int fco_key_similarity_columns(const void* K_cand, int dtype, int n_heads,
+                               int L_k, int d, int64_t k_hs, int64_t k_rs,
+                               const int32_t* cols, int n_cols, int red_mode,
+                               double* out, int n_threads);
+
+/* The softmax argument of Eq. 11 for chosen columns only, by its plain
+ * definition: out[h][c] = (1/L_k) sum_{i != j} khat_i . khat_j for j = cols[c]
+ * (red_mode PLAIN) or max_{i != j} khat_i . khat_j (MAXSIM).  K_cand is
+ * [n_heads, L_k, d] with strides k_hs, k_rs; out is [n_heads, n_cols]. */
+int fco_key_similarity_columns(const void* K_cand, int dtype, int n_heads,
+                               int L_k, int d, int64_t k_hs, int64_t k_rs,
+                               const int32_t* cols, int n_cols, int red_mode,
+                               double* out, int n_threads);
 
 /* Per-head top-B (Sec. 3.3, text after Eq. 12) and retention of the selected
  * K/V rows.  Total order: score descending, index ascending; NaN ranks as

@@ -482,3 +482,49 @@ def test_cache_apply_matches_library_arithmetic_and_rounding():
     # a zero residual serves the input back unchanged; an empty chunk is fine
     y, _ = oracle.chunk_cache_apply(xf.numpy(), yf.numpy(), np.zeros(n, np.float32), [0, 0, n], [0, 0])
     assert np.array_equal(y, xf.numpy())
+
+
+# --------------------------------------------------------------------------- similarity statistics beyond Eq. 11
+
+def test_max_similarity_mode_against_library_routines_and_closed_forms():
+    # torch fp64: normalise, cosine matrix, diagonal excluded, column maximum, softmax over tokens
+    H, L, d = 2, 60, 16
+    K = wl.normal((H, L, d), 801, 1.0)
+    K[1, 7] = K[1, 3] * 2.5          # a duplicated direction: both tokens get similarity 1
+    Q = wl.normal((H, 5, d), 802, 1.0)
+    out = oracle.kv_score(Q.numpy(), K.numpy(), red_mode=oracle.RED_MAXSIM, lambda_=0.0)
+    Kh = torch.nn.functional.normalize(K.double(), dim=-1)
+    S = Kh @ Kh.transpose(1, 2)
+    S[:, torch.arange(L), torch.arange(L)] = -float("inf")
+    a = S.max(dim=1).values
+    np.testing.assert_allclose(out["red"], torch.softmax(a, dim=-1).numpy(), rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(oracle.key_similarity_columns(K.numpy(), np.arange(L), oracle.RED_MAXSIM), a.numpy(),
+                               rtol=1e-12, atol=1e-15)
+    assert abs(a[1, 7].item() - 1.0) < 1e-12 and abs(a[1, 3].item() - 1.0) < 1e-12
+    # mutually orthogonal keys: every maximum is 0 -> uniform Red; the mean-based Eq. 11 gives uniform Red too
+    E = torch.eye(8).reshape(1, 8, 8) * torch.arange(1, 9).reshape(1, 8, 1)
+    out = oracle.kv_score(Q[:1, :, :8].contiguous().numpy(), E.numpy(), red_mode=oracle.RED_MAXSIM)
+    np.testing.assert_allclose(out["red"], np.full((1, 8), 1 / 8), rtol=1e-12)
+    # the maximum is never below the mean of the other columns' similarities, and differs from it in general
+    mean_cols = oracle.key_similarity_columns(K.numpy(), np.arange(L), oracle.RED_PLAIN)
+    assert (a.numpy() >= mean_cols * L / (L - 1) - 1e-12).all() and np.abs(a.numpy() - mean_cols).max() > 0.1
+
+
+def test_similarity_columns_match_the_full_matrix_and_the_mean_key_identity():
+    # sampled columns of the plain definition = the same columns of the full evaluation (both red modes of
+    # kv_score), also for bf16 storage, a zero key and strided sampling
+    H, L, d = 3, 130, 32
+    K = wl.normal((H, L, d), 811, 0.7, torch.bfloat16)
+    K[2, 11] = 0
+    Q = wl.normal((H, 4, d), 812, 0.7, torch.bfloat16)
+    cols = np.array([0, 1, 11, 64, 129], np.int32)
+    a_cols = oracle.key_similarity_columns(wl.bits(K), cols, oracle.RED_PLAIN)
+    Kh = K.double() / K.double().norm(dim=-1, keepdim=True).clamp_min(1e-12)
+    S = Kh @ Kh.transpose(1, 2)
+    S[:, torch.arange(L), torch.arange(L)] = 0.0
+    np.testing.assert_allclose(a_cols, S.mean(dim=1)[:, cols].numpy(), rtol=1e-12, atol=1e-15)
+    # and Red of the two modes of kv_score is the softmax of exactly these arguments
+    full = oracle.key_similarity_columns(wl.bits(K), np.arange(L), oracle.RED_PLAIN)
+    for mode in (oracle.RED_PLAIN, oracle.RED_MEANKEY):
+        red = oracle.kv_score(wl.bits(Q), wl.bits(K), red_mode=mode)["red"]
+        np.testing.assert_allclose(red, torch.softmax(torch.from_numpy(full), dim=-1).numpy(), rtol=1e-10)

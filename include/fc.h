@@ -31,6 +31,9 @@
  *   - The library keeps no state between calls except immutable per-device
  *     attributes inside fc_ctx.  Calls on different streams may overlap as long
  *     as their buffers and workspaces do not.
+ *   - One exception to the two points above: fc_chunk_decide_static takes no
+ *     workspace; its scratch is an array inside the library that all its calls
+ *     on a device share (see its comment for what that implies).
  */
 #ifndef FC_H_
 #define FC_H_
@@ -55,6 +58,9 @@ typedef enum {
 } fc_status;
 
 typedef enum { FC_BF16 = 0, FC_F32 = 1 } fc_dtype;
+
+/* Reuse policy of fc_chunk_decide: the paper's chunkwise rule, or the uniform policy it compares with. */
+typedef enum { FC_POLICY_CHUNKWISE = 0, FC_POLICY_UNIFORM = 1 } fc_policy;
 
 /* Bits of the device status word. */
 enum {
@@ -89,6 +95,13 @@ int fc_sm_count(const fc_ctx* ctx);
  *     acc_i <- 0 if recompute_i else s_i
  * A zero denominator yields r = +inf if the numerator is positive, else 0.
  *
+ * policy = FC_POLICY_UNIFORM is the "traditional reuse" the paper compares with (caption of Fig. 3): all chunks of
+ * a step share one compute / reuse status, except chunks that must be computed anyway (chunk_step[i] < warmup_m
+ * or force[i]: a newly initialised chunk).  Over the sharing chunks S taken as one tensor (Eq. 4):
+ *     r = sum_S |cur - prev| / sum_S |prev|,   s = acc[first chunk of S] + r   (fp32)
+ *     recompute_i = (i not in S) || s > eps;   every acc[i] <- 0 if s > eps (or S is empty) else s
+ * and l1rel[i] = r for i in S, the chunk's own indicator otherwise.
+ *
  *   cur, prev        DEVICE, `dtype` elements; chunk i occupies elements
  *                    [chunk_elem_off[i], chunk_elem_off[i+1]) of both.  The vectorised path
  *                    is taken when every offset is a multiple of 16 bytes.
@@ -107,7 +120,7 @@ int fc_sm_count(const fc_ctx* ctx);
 size_t fc_chunk_decide_workspace_bytes(int64_t total_elems, int n_chunks);
 int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
                     const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
-                    int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
+                    int warmup_m, float eps, const uint8_t* force, int policy, float* acc, float* l1rel,
                     uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
                     uint32_t* status, void* ws, size_t ws_bytes);
 
@@ -134,9 +147,32 @@ int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const void* prev
 size_t fc_chunk_decide_static_max_bytes(void);
 int fc_chunk_decide_static(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
                            const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
-                           int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
+                           int warmup_m, float eps, const uint8_t* force, int policy, float* acc, float* l1rel,
                            uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
                            uint32_t* status);
+
+/* ------------------------------------------------------------------------------------------
+ * fc_chunk_cache_apply — serving the chunks that were not recomputed from the activation cache.
+ *
+ * Paper (Sec. 3.2, text after Eq. 8): when the rule says reuse, the chunk's cached activations are
+ * reused instead of a forward pass; the cache is one tensor the size of the model input (efficiency
+ * appendix).  The cache holds, per chunk, the residual output - input of the chunk's last computed
+ * forward; a reused chunk's output is its current input plus that residual.  For every element e of
+ * chunk i (flat layout as in fc_chunk_decide):
+ *     recompute[i] != 0:  cache[e] <- y[e] - x[e]       (y holds the fresh output of the forward)
+ *     recompute[i] == 0:  y[e]     <- x[e] + cache[e]   (the cache is left as it is)
+ * in fp32, rounded once to `dtype` (round to nearest even for bf16).  Call it after the forward of
+ * the active chunks, with the recompute flags fc_chunk_decide left on the device.
+ *
+ *   x_in             DEVICE, `dtype`: the chunks' inputs at this step.
+ *   y_io             DEVICE, `dtype`, in/out: outputs; only skipped chunks are written.
+ *   cache            DEVICE, `dtype`, in/out: only computed chunks are written.
+ *   chunk_elem_off   HOST [n_chunks+1]; recompute DEVICE [n_chunks].
+ * The three tensors must not overlap.  Needs no workspace.  Moves 3 x (elements x element size)
+ * bytes with 16-byte accesses when every offset is a multiple of 16 bytes. */
+int fc_chunk_cache_apply(fc_ctx* ctx, void* stream, const void* x_in, void* y_io, void* cache, int dtype,
+                         const int64_t* chunk_elem_off, int n_chunks, const uint8_t* recompute,
+                         uint32_t* status);
 
 /* ------------------------------------------------------------------------------------------
  * fc_chunk_attention — chunk-causal attention of the active chunks.
@@ -159,8 +195,8 @@ typedef struct {
   int64_t o_hs, o_rs;
   int64_t kv_rows;                           /* physical rows per head in the K/V store */
   float scale;                               /* 0 => 1/sqrt(d) */
-  int32_t impl;                              /* 0 auto; 1 force the CUDA-core kernel; 2 force tcgen05
-                                                (warp-specialised); 3 force the single-stage tcgen05 kernel */
+  int32_t impl;                              /* 0 auto; 1 force the CUDA-core kernel; 2 force the tcgen05
+                                                kernel (FC_ERR_UNSUPPORTED where it does not apply) */
 } fc_attn_desc;
 
 /*   Q, O             DEVICE [H_q, rows, d]; K, V DEVICE [H_kv, kv_rows, d]; `dtype` elements.

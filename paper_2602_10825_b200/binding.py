@@ -14,6 +14,7 @@ _LIB_PATH = os.path.join(_PKG, "libfc.so")
 _HEADER = os.path.join(_ROOT, "include", "fc.h")
 
 BF16, F32 = 0, 1
+POLICY_CHUNKWISE, POLICY_UNIFORM = 0, 1
 STATUS_BITS = {"timeout": 1, "nan_score": 2, "bad_index": 4}
 
 
@@ -154,7 +155,7 @@ class Context:
 
     # ------------------------------------------------------------------ fc_chunk_decide
     def chunk_decide(self, cur, prev, chunk_elem_off, chunk_step, warmup_m, eps, acc, *, force=None,
-                     l1rel=None, recompute=None, active_ids=None, n_active=None, status=None, ws=None):
+                     policy=POLICY_CHUNKWISE, l1rel=None, recompute=None, active_ids=None, n_active=None, status=None, ws=None):
         off = np.ascontiguousarray(np.asarray(chunk_elem_off, dtype=np.int64))
         n = len(off) - 1
         dev = cur.device
@@ -167,7 +168,7 @@ class Context:
         rc = self._L.fc_chunk_decide(
             self._h, self._stream(), _dev(cur, "cur"), _dev(prev, "prev"), _dt(cur),
             off.ctypes.data_as(C.c_void_p), n, _dev(chunk_step, "chunk_step", torch.int32), int(warmup_m),
-            C.c_float(eps), _dev(force, "force", torch.uint8), _dev(acc, "acc", torch.float32),
+            C.c_float(eps), _dev(force, "force", torch.uint8), int(policy), _dev(acc, "acc", torch.float32),
             _dev(l1rel, "l1rel", torch.float32), _dev(recompute, "recompute", torch.uint8),
             _dev(active_ids, "active_ids", torch.int32), _dev(n_active, "n_active", torch.int32),
             _dev(status, "status", torch.int32), _dev(ws, "ws"), C.c_size_t(ws.numel()))
@@ -175,7 +176,7 @@ class Context:
         return dict(l1rel=l1rel, recompute=recompute, active_ids=active_ids, n_active=n_active, acc=acc)
 
     def chunk_decide_static(self, cur, prev, chunk_elem_off, chunk_step, warmup_m, eps, acc, *, l1rel, recompute,
-                            active_ids, n_active, force=None, status=None):
+                            active_ids, n_active, force=None, policy=POLICY_CHUNKWISE, status=None):
         """fc_chunk_decide_static: the decision without a workspace, for callers that cannot allocate device
         memory (the scratch is a fixed 1 MiB array inside the library).  Every output tensor is passed in, so
         this wrapper allocates nothing on the device either."""
@@ -184,12 +185,27 @@ class Context:
         rc = self._L.fc_chunk_decide_static(
             self._h, self._stream(), _dev(cur, "cur"), _dev(prev, "prev"), _dt(cur),
             off.ctypes.data_as(C.c_void_p), n, _dev(chunk_step, "chunk_step", torch.int32), int(warmup_m),
-            C.c_float(eps), _dev(force, "force", torch.uint8), _dev(acc, "acc", torch.float32),
+            C.c_float(eps), _dev(force, "force", torch.uint8), int(policy), _dev(acc, "acc", torch.float32),
             _dev(l1rel, "l1rel", torch.float32), _dev(recompute, "recompute", torch.uint8),
             _dev(active_ids, "active_ids", torch.int32), _dev(n_active, "n_active", torch.int32),
             _dev(status, "status", torch.int32))
         self._check(rc, "fc_chunk_decide_static")
         return dict(l1rel=l1rel, recompute=recompute, active_ids=active_ids, n_active=n_active, acc=acc)
+
+    # ------------------------------------------------------------------ fc_chunk_cache_apply
+    def chunk_cache_apply(self, x_in, y_io, cache, chunk_elem_off, recompute, *, status=None):
+        off = np.ascontiguousarray(np.asarray(chunk_elem_off, dtype=np.int64))
+        if not (x_in.dtype == y_io.dtype == cache.dtype):
+            raise FcError("x_in, y_io and cache must share one dtype")
+        for name, t in (("x_in", x_in), ("y_io", y_io), ("cache", cache)):
+            if not t.is_contiguous() or t.numel() < int(off[-1]):
+                raise FcError(f"{name} must be contiguous and hold every chunk's elements")
+        rc = self._L.fc_chunk_cache_apply(
+            self._h, self._stream(), _dev(x_in, "x_in"), _dev(y_io, "y_io"), _dev(cache, "cache"), _dt(x_in),
+            off.ctypes.data_as(C.c_void_p), len(off) - 1, _dev(recompute, "recompute", torch.uint8),
+            _dev(status, "status", torch.int32))
+        self._check(rc, "fc_chunk_cache_apply")
+        return y_io, cache
 
     # ------------------------------------------------------------------ fc_chunk_attention
     def chunk_attention(self, Q, K, V, q_chunk_row_off, kv_visible_len, seg_logical_off, seg_phys_off,

@@ -23,7 +23,8 @@ extern "C" int fc_chunk_attention(fc_ctx* ctx, void* stream, const fc_attn_desc*
   if (desc->H_q <= 0 || desc->H_kv <= 0 || desc->H_q % desc->H_kv || desc->W <= 0 || desc->kv_rows <= 0)
     return FC_ERR_INVALID_ARG;
   if (desc->W > FC_MAX_CHUNKS) return FC_ERR_UNSUPPORTED;
-  if (desc->impl < 0 || desc->impl > 3) return FC_ERR_INVALID_ARG;
+  if (desc->impl < 0 || desc->impl > 2) return FC_ERR_INVALID_ARG;
+  if (!(desc->scale >= 0.f)) return FC_ERR_INVALID_ARG;  // 0 selects 1/sqrt(d); the kernels assume a positive scale
   if (!kv_token_index) {
     if (!seg_logical_off || !seg_phys_off || n_seg <= 0) return FC_ERR_INVALID_ARG;
     if (n_seg > FC_MAX_SEGMENTS) return FC_ERR_UNSUPPORTED;
@@ -78,6 +79,6 @@ extern "C" int fc_chunk_attention(fc_ctx* ctx, void* stream, const fc_attn_desc*
   cudaStream_t st = (cudaStream_t)stream;
   const bool tc_ok = fc::attention_tc_supported(g, dtype);
   if (desc->impl >= 2 && !tc_ok) return FC_ERR_UNSUPPORTED;
-  if (desc->impl != 1 && tc_ok) return fc::attention_tc(ctx, st, g, Q, K, V, O, ws, ws_bytes, desc->impl == 3);
+  if (desc->impl != 1 && tc_ok) return fc::attention_tc(ctx, st, g, Q, K, V, O, ws, ws_bytes);
   return fc::attention_simt(st, g, Q, K, V, dtype, O);
 }

@@ -24,11 +24,9 @@ struct AttnGeom {
 
 int attention_simt(cudaStream_t st, const AttnGeom& g, const void* Q, const void* K, const void* V,
                    int dtype, void* O);
-// bf16 only, segment-table addressing only.
-// `basic` selects the single-stage kernel (one CTA per tile, no warp roles) instead of the
-// warp-specialised one.
+// bf16 only: builds the tensor maps and launches the warp-specialised tcgen05 kernel.
 int attention_tc(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const void* Q, const void* K,
-                 const void* V, void* O, void* ws, size_t ws_bytes, bool basic);
+                 const void* V, void* O, void* ws, size_t ws_bytes);
 size_t attention_tc_workspace_bytes();
 // warp-specialised kernel; tensor maps as built by attention_tc, `counter` = 4 bytes of workspace
 int attention_ws_launch(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const CUtensorMap& tq,

@@ -10,6 +10,7 @@
 //                                    other warps through a 2-slot ring, then loads the Q pair and
 //                                    streams K and V tiles into 2-stage rings
 //   warps 9,10 MMA issuers           one thread per query tile
+//   warp  11   tail patcher          zeroes the rows of a V stage that lie past the end of a segment
 // Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
 // A key tile of 128 tokens is worked through as two halves of 64: S_x is two 64-column accumulators, each with
 // its own "full" and "P ready" barriers, and P (bf16) of a half overwrites the first 32 columns of that half.
@@ -33,6 +34,12 @@
 // cubic): 900 clocks per half tile in isolation; a larger share costs more fma-pipe time than it saves.
 // As measured with clock probes, a softmax warp now spends about 75 % of its time in exponentials and 10 % waiting
 // for S; the tensor pipe has work about 75 % of the time.
+// Tails.  A segment's last key tile may be ragged: the TMA box still brings 128 physical rows, and the rows past the
+// segment's end are whatever the K/V store holds there (another segment, or slots of the buffer that were never
+// written).  Their logits are replaced by -inf before the row maximum and their P is exactly 0 (a ragged half takes
+// every exponential on the special-function unit, and masked columns are forced to 0); the V rows themselves are
+// overwritten with zeros in shared memory by warp 11 before the PV instructions of that tile are issued, so that not
+// even a NaN or an infinity in such a row can reach an output (0 x inf would).
 // Every mbarrier wait is bounded (see mbar_wait_bounded); tensor memory is always released.
 #include <cmath>
 
@@ -53,23 +60,17 @@ constexpr float kRescaleThreshold = 8.f;  // log2 units
 // Registers per thread after the split: softmax warpgroups / the warpgroup of the copy and MMA warps.
 // The CTA owns 384 x 168 registers from launch (168 = what the launch bounds allow); setmaxnreg only moves
 // registers inside that pool, and an increase that the pool cannot cover would wait forever.
-#ifndef FC_ATTN_REGS_HI
-#define FC_ATTN_REGS_HI 200
-#define FC_ATTN_REGS_LO 104
-#endif
-static_assert(256 * FC_ATTN_REGS_HI + 128 * FC_ATTN_REGS_LO <= 384 * 168, "register split exceeds the CTA's pool");
-static_assert(FC_ATTN_REGS_HI % 8 == 0 && FC_ATTN_REGS_LO % 8 == 0, "setmaxnreg takes multiples of 8");
-// of every four column pairs, how many take their exponential on the fma pipe instead of the special-function unit
-#ifndef FC_ATTN_POLY_OF_4
-#define FC_ATTN_POLY_OF_4 1
-#endif
-constexpr int kPolyOf4 = FC_ATTN_POLY_OF_4;
-#define FC_STR2(x) #x
-#define FC_STR(x) FC_STR2(x)
+constexpr int kRegsHi = 200, kRegsLo = 104;
+static_assert(256 * kRegsHi + 128 * kRegsLo <= 384 * 168, "register split exceeds the CTA's pool");
+static_assert(kRegsHi % 8 == 0 && kRegsLo % 8 == 0, "setmaxnreg takes multiples of 8");
+// Of every four column pairs, how many take their exponential on the fma pipe instead of the special-function unit
+// (measured: 0 -> 1115 clocks per half tile per warp, 1 -> 900, 2 -> 970, 4 -> 1410).
+constexpr int kPolyOf4 = 1;
 
 struct WsSmem {
   uint64_t q_full, q_empty;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  uint64_t v_fixed[kStages];             // the tail patcher is done with the stage (one phase per tile, like v_full)
   uint64_t s_full[2][2], p_ready[2][2];  // [query tile][half of the key tile]
   uint64_t pv_done[2];                   // per query tile: one phase per PV half, in issue order
   uint64_t o_done[2];                    // per query tile: one phase per item, after its last PV
@@ -88,8 +89,11 @@ struct Item {
 };
 
 // P = 2^(S * scale - m) for one row of a 64-column half tile, written as bf16 to tensor-memory columns
-// [t_p, t_p + 32); returns the row sum.
-__device__ __forceinline__ float exp_half(const uint32_t (&sv)[kHalf], float scale_log2, float m, uint32_t t_p) {
+// [t_p, t_p + 32); returns the row sum.  kRagged: only the first n_valid columns are visible; the others get P = 0
+// exactly and every exponential is taken on the special-function unit (2^-inf = 0 there, 2^-125 on the fma pipe).
+template <bool kRagged>
+__device__ __forceinline__ float exp_half(const uint32_t (&sv)[kHalf], float scale_log2, float m, uint32_t t_p,
+                                          int n_valid) {
   const uint64_t sc2 = pack2(scale_log2, scale_log2), nm2 = pack2(-m, -m);
   uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
@@ -100,7 +104,7 @@ __device__ __forceinline__ float exp_half(const uint32_t (&sv)[kHalf], float sca
       const uint64_t x = fma2(pack2(__uint_as_float(sv[q2 * 32 + 2 * i]), __uint_as_float(sv[q2 * 32 + 2 * i + 1])),
                               sc2, nm2);
       float p0, p1;
-      if (kPolyOf4 > 0 && (i & 3) >= 4 - kPolyOf4) {
+      if (!kRagged && kPolyOf4 > 0 && (i & 3) >= 4 - kPolyOf4) {
         // the special-function unit is what bounds the softmax warps: a share of the pairs goes to the fma pipe
         ex2_fma_pair(x, p0, p1);
       } else {
@@ -108,6 +112,10 @@ __device__ __forceinline__ float exp_half(const uint32_t (&sv)[kHalf], float sca
         unpack2(x, x0, x1);
         p0 = ex2(x0);
         p1 = ex2(x1);
+      }
+      if (kRagged) {
+        if (q2 * 32 + 2 * i >= n_valid) p0 = 0.f;
+        if (q2 * 32 + 2 * i + 1 >= n_valid) p1 = 0.f;
       }
       sum2[i & 1] = add2(sum2[i & 1], pack2(p0, p1));
       pk[i] = cvt_bf16x2(p0, p1);
@@ -150,7 +158,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       mbar_init(smem_u32(&sh->k_full[s]), 1);
       mbar_init(smem_u32(&sh->k_empty[s]), 2);  // both MMA threads
       mbar_init(smem_u32(&sh->v_full[s]), 1);
-      mbar_init(smem_u32(&sh->v_empty[s]), 2);
+      mbar_init(smem_u32(&sh->v_empty[s]), 3);  // both MMA threads and the tail patcher
+      mbar_init(smem_u32(&sh->v_fixed[s]), 1);
     }
     for (int x = 0; x < 2; ++x) {
       for (int u = 0; u < 2; ++u) {
@@ -160,7 +169,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       mbar_init(smem_u32(&sh->pv_done[x]), 1);
       mbar_init(smem_u32(&sh->o_done[x]), 1);
       mbar_init(smem_u32(&sh->it_full[x]), 1);
-      mbar_init(smem_u32(&sh->it_empty[x]), 10);  // the two MMA threads and the eight softmax warps
+      mbar_init(smem_u32(&sh->it_empty[x]), 11);  // the two MMA threads, the eight softmax warps, the tail patcher
       sh->it_slot[x] = -1;
     }
     mbar_fence_init();
@@ -242,7 +251,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   // Registers move from the third warpgroup, which only issues copies and MMAs, to the softmax
   // warpgroups, which hold a 128-column row of S per thread.
   if (warp >= 8) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 " FC_STR(FC_ATTN_REGS_LO) ";");
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLo));
   if (warp == 8) {
     // ------------------------------------------------------------------ scheduler + TMA producer
     uint32_t kv = 0, it_n = 0;
@@ -334,6 +343,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     // barrier addresses as plain registers: the issue loop should be little more than the MMAs themselves
     const uint32_t b_kfull = smem_u32(&sh->k_full[0]), b_kempty = smem_u32(&sh->k_empty[0]);
     const uint32_t b_vfull = smem_u32(&sh->v_full[0]), b_vempty = smem_u32(&sh->v_empty[0]);
+    const uint32_t b_vfixed = smem_u32(&sh->v_fixed[0]);
     const uint32_t b_sfull = smem_u32(&sh->s_full[x][0]), b_pready = smem_u32(&sh->p_ready[x][0]);
     const uint32_t b_pvdone = smem_u32(&sh->pv_done[x]);
     // Barrier phases are counted per use: tile B sits out the items in which it has no rows (the last item of a
@@ -374,13 +384,22 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         umma_commit(b_sfull + 8);
         umma_commit(b_kempty + 8 * st);
       }
+      // the walk over the segments, to know which tiles are ragged (their V stage is patched before PV)
+      int seg = 0, seg_left = n_tiles > 0 ? min(g.seg_log[1], it.n_vis) - g.seg_log[0] : 0;
       for (int j = 0; j < n_tiles; ++j, ++kv, ++uses) {
         const uint32_t st = kv & 1, ph = (kv >> 1) & 1;
         const uint32_t st2 = st ^ 1, ph2 = ((kv + 1) >> 1) & 1;  // the next key tile's stage
         const bool more = j + 1 < n_tiles;
+        const bool ragged = seg_left < kBN;
+        seg_left -= kBN;
+        if (seg_left <= 0 && more) {
+          ++seg;
+          seg_left = min(g.seg_log[seg + 1], it.n_vis) - g.seg_log[seg];
+        }
         prep_pv(st, 0);
         if (more) prep_s(st2, 0);
         mbar_wait_bounded(b_vfull + 8 * st, ph, abort);
+        if (ragged) mbar_wait_bounded(b_vfixed + 8 * st, ph, abort);
         mbar_wait_bounded(b_pready, uses & 1, abort);
         tc_fence_after();
         issue_pv(j > 0);
@@ -408,9 +427,46 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       umma_commit(smem_u32(&sh->o_done[x]));
     }
     }
+  } else {
+    // ------------------------------------------------------------------ tail patcher (warp 11)
+    // Follows the V ring tile by tile.  On a ragged tile it writes zeros over the rows past the segment's end
+    // (row r of a stage is 128 bytes at r * 128 in every 64-column block, whatever the swizzle does inside them),
+    // makes the writes visible to the tensor cores' proxy and only then reports the stage as fixed.  It takes
+    // part in the ring's flow control (v_empty), so the copy warp cannot refill a stage that is being patched and
+    // the phases of v_fixed stay in step with those of v_full.
+    uint8_t* v_tiles = smem + (2 + kStages) * kTileBytes;
+    uint32_t kv = 0;
+    for (uint32_t it_n = 0;; ++it_n) {
+      const int item = next_item(it_n);
+      if (item < 0) break;
+      const Item it = decode(item);
+      for (int s = 0; s < g.n_seg; ++s) {
+        const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
+        if (seg_vis <= 0) break;
+        for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv) {
+          const int st = kv % kStages, ph = (kv / kStages) & 1;
+          const int cols_valid = min(kBN, seg_vis - j0);
+          warp_wait(smem_u32(&sh->v_full[st]), ph, abort);
+          if (cols_valid < kBN) {
+            uint8_t* vt = v_tiles + st * kTileBytes;
+            const int n16 = (kBN - cols_valid) * kAtoms * 8;  // 16-byte pieces to clear
+            for (int i = lane; i < n16; i += 32) {
+              const int r = cols_valid + i / (kAtoms * 8), x = (i / 8) % kAtoms, c = i % 8;
+              *reinterpret_cast<uint4*>(vt + x * kAtomBytes + r * 128 + c * 16) = make_uint4(0u, 0u, 0u, 0u);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          }
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(smem_u32(&sh->v_fixed[st]));
+            mbar_arrive(smem_u32(&sh->v_empty[st]));
+          }
+        }
+      }
+    }
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 " FC_STR(FC_ATTN_REGS_HI) ";");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsHi));
     // ------------------------------------------------------------------ softmax + epilogue, tile x
     const int x = warp >> 2;
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
@@ -490,7 +546,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
               wait_pv();
               rescale_o(alpha);
             }
-            const float row_sum = exp_half(sv, scale_log2, m, t_su);  // masked columns: 2^-inf = 0 (2^-125 on the fma pipe)
+            const float row_sum = mine_valid < kHalf ? exp_half<true>(sv, scale_log2, m, t_su, mine_valid)
+                                                     : exp_half<false>(sv, scale_log2, m, t_su, kHalf);
             l = l * alpha + row_sum;
             tmem_wait_st();
             tc_fence_before();

@@ -40,6 +40,28 @@ inline int elem_size(int dtype) { return dtype == FC_F32 ? 4 : 2; }
     }                                               \
   } while (0)
 
+// Programmatic dependent launch.  launch_pdl() starts `kernel` so that its blocks may become resident while the
+// previous kernel of the stream is still running (once every block of that kernel has executed
+// pdl_launch_dependents() or exited); the kernel must execute pdl_wait() before it reads or writes anything the
+// previous kernel touches: the wait returns when that kernel has completed and its writes are visible.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // Storage element -> float.
 template <typename T> __device__ __forceinline__ float to_float(T x);
 template <> __device__ __forceinline__ float to_float<float>(float x) { return x; }

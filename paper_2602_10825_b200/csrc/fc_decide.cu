@@ -1,12 +1,16 @@
 // fc_chunk_decide: per-chunk relative-L1 indicator (Eq. 5) and the accumulate / threshold /
-// reset rule (Eq. 8).
+// reset rule (Eq. 8); as a switch, the uniform policy the paper compares with (caption of Fig. 3): one shared
+// decision for all chunks of a step except those that must be computed anyway.
 //
-// Two launches.  (1) A streaming segmented reduction: the chunks are cut into slabs of 16 KiB
+// Two launches, the second one programmatically dependent on the first (it is scheduled under the first one's
+// tail and waits there).  (1) A streaming segmented reduction: the chunks are cut into slabs of 16 KiB
 // per tensor, one block per slab; every thread sums |cur-prev| and |prev| of 4 interleaved
 // 16-byte vectors in fp32, the block combines them in fp64 in a fixed tree and writes one
 // (num, den) pair per slab.  (2) One block: a warp per chunk adds that chunk's slab pairs in a
 // fixed order in fp64, forms r, applies the rule in fp32 and compacts the active ids.
 // No atomics: results are bit-reproducible from run to run.
+#include <atomic>
+
 #include "fc_common.cuh"
 
 namespace {
@@ -50,6 +54,7 @@ decide_partial_kernel(const T* __restrict__ cur, const T* __restrict__ prev, Dec
                       double2* __restrict__ partial) {
   constexpr int kElemPerVec = 16 / (int)sizeof(T);
   constexpr int kSlabElems = kSlabBytes / (int)sizeof(T);
+  fc::pdl_launch_dependents();  // the finalising block may take its place on an SM; it waits for this grid to end
   const int b = blockIdx.x;
   int c = 0;
   while (c + 1 < g.n_chunks && b >= g.slab_off[c + 1]) ++c;
@@ -97,14 +102,22 @@ decide_partial_kernel(const T* __restrict__ cur, const T* __restrict__ prev, Dec
   }
 }
 
+// Eq. 5's ratio; a zero denominator yields +inf if anything changed, else 0
+__device__ __forceinline__ double ratio(double num, double den) {
+  if (den > 0.0) return num / den;
+  return num > 0.0 ? (double)INFINITY : 0.0;
+}
+
 __global__ void __launch_bounds__(1024)
 decide_finalize_kernel(DecideGeom g, const double2* __restrict__ partial,
                        const int32_t* __restrict__ chunk_step, int warmup_m, float eps,
-                       const uint8_t* __restrict__ force, float* __restrict__ acc,
+                       const uint8_t* __restrict__ force, int policy, float* __restrict__ acc,
                        float* __restrict__ l1rel, uint8_t* __restrict__ recompute,
                        int32_t* __restrict__ active_ids, int32_t* __restrict__ n_active) {
   __shared__ uint8_t flag[FC_MAX_CHUNKS];
   __shared__ double2 part[32];
+  __shared__ double2 chunk_sum[FC_MAX_CHUNKS];  // uniform policy: every chunk's (num, den)
+  fc::pdl_wait();  // launched under the reduction's tail: its slab pairs are complete and visible from here on
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // The 32 warps are shared out over the chunks, a power of two of them per chunk (all 32 for one chunk, one each
   // for 32 or more): every warp adds up a fixed subset of the chunk's slabs, the warps of a chunk are combined in
@@ -135,22 +148,52 @@ decide_finalize_kernel(DecideGeom g, const double2* __restrict__ partial,
         num += part[warp + w].x;
         den += part[warp + w].y;
       }
-      double r;
-      if (den > 0.0)
-        r = num / den;
-      else
-        r = num > 0.0 ? (double)INFINITY : 0.0;
-      const float rf = (float)r;
-      const float s = __fadd_rn(acc[c], rf);
-      const bool rec = chunk_step[c] < warmup_m || (force && force[c]) || s > eps;
-      if (l1rel) l1rel[c] = rf;
-      recompute[c] = rec ? 1 : 0;
-      acc[c] = rec ? 0.f : s;
-      flag[c] = rec ? 1 : 0;
+      if (policy == FC_POLICY_UNIFORM) {
+        chunk_sum[c] = make_double2(num, den);
+      } else {
+        const float rf = (float)ratio(num, den);
+        const float s = __fadd_rn(acc[c], rf);
+        const bool rec = chunk_step[c] < warmup_m || (force && force[c]) || s > eps;
+        if (l1rel) l1rel[c] = rf;
+        recompute[c] = rec ? 1 : 0;
+        acc[c] = rec ? 0.f : s;
+        flag[c] = rec ? 1 : 0;
+      }
     }
     __syncthreads();  // part[] is reused by the next round
   }
   __syncthreads();
+  if (threadIdx.x == 0 && policy == FC_POLICY_UNIFORM) {
+    // One decision for the chunks that share it (those neither in warm-up nor forced): Eq. 4 over them as one
+    // tensor, sums taken in chunk order, then Eq. 8 on the shared accumulator (read from the first sharing chunk,
+    // written to every entry so that they stay equal).
+    double num = 0.0, den = 0.0;
+    int first = -1;
+    for (int c = 0; c < g.n_chunks; ++c) {
+      const bool own = chunk_step[c] < warmup_m || (force && force[c]);
+      flag[c] = own ? 2 : 0;
+      if (own) continue;
+      if (first < 0) first = c;
+      num += chunk_sum[c].x;
+      den += chunk_sum[c].y;
+    }
+    bool shared_compute = true;
+    float acc_next = 0.f, r_shared = 0.f;
+    if (first >= 0) {
+      r_shared = (float)ratio(num, den);
+      const float s = __fadd_rn(acc[first], r_shared);
+      shared_compute = s > eps;
+      acc_next = shared_compute ? 0.f : s;
+    }
+    for (int c = 0; c < g.n_chunks; ++c) {
+      const bool own = flag[c] == 2;
+      if (l1rel) l1rel[c] = own ? (float)ratio(chunk_sum[c].x, chunk_sum[c].y) : r_shared;
+      const bool rec = own || shared_compute;
+      recompute[c] = rec ? 1 : 0;
+      acc[c] = acc_next;
+      flag[c] = rec ? 1 : 0;
+    }
+  }
   if (threadIdx.x == 0) {
     int n = 0;
     for (int c = 0; c < g.n_chunks; ++c)
@@ -173,10 +216,11 @@ extern "C" size_t fc_chunk_decide_workspace_bytes(int64_t total_elems, int n_chu
 
 extern "C" int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
                                const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
-                               int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
-                               uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
+                               int warmup_m, float eps, const uint8_t* force, int policy, float* acc,
+                               float* l1rel, uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
                                uint32_t* status, void* ws, size_t ws_bytes) {
   (void)status;
+  if (policy != FC_POLICY_CHUNKWISE && policy != FC_POLICY_UNIFORM) return FC_ERR_INVALID_ARG;
   if (!ctx || !chunk_elem_off || !chunk_step || !acc || !recompute || !active_ids || !n_active)
     return FC_ERR_INVALID_ARG;
   if (n_chunks <= 0) return FC_ERR_INVALID_ARG;
@@ -223,9 +267,9 @@ extern "C" int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const
     }
     FC_LAUNCH_CHECK("decide_partial_kernel");
   }
-  decide_finalize_kernel<<<1, 1024, 0, st>>>(g, partial, chunk_step, warmup_m, eps, force, acc, l1rel,
-                                             recompute, active_ids, n_active);
-  FC_LAUNCH_CHECK("decide_finalize_kernel");
+  FC_CUDA_CHECK(fc::launch_pdl(decide_finalize_kernel, dim3(1), dim3(1024), 0, st, g, (const double2*)partial,
+                               chunk_step, warmup_m, eps, force, policy, acc, l1rel, recompute, active_ids,
+                               n_active));
   return FC_OK;
 }
 
@@ -241,14 +285,16 @@ constexpr size_t kStaticScratchBytes = 1u << 20;  // 65,536 slabs of 16 KiB per 
 static __device__ __align__(256) unsigned char g_decide_scratch[kStaticScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {};  // device address of g_decide_scratch on each device (0 = not looked up)
+// device address of g_decide_scratch on each device (null = not looked up yet)
+std::atomic<void*> g_scratch_addr[kMaxDevices];
 
 // Look the address up on first use per device.  Not an allocation: the array is part of the
 // module image every device already holds.  Concurrent first calls may both do the lookup; they
-// get the same answer.
+// get the same answer and store the same value.
 int static_scratch(int device, void** out) {
   if (device < 0 || device >= kMaxDevices) return FC_ERR_UNSUPPORTED;
-  if (!g_scratch_addr[device]) {
+  void* known = g_scratch_addr[device].load(std::memory_order_acquire);
+  if (!known) {
     int current = -1;
     FC_CUDA_CHECK(cudaGetDevice(&current));
     if (current != device) FC_CUDA_CHECK(cudaSetDevice(device));
@@ -259,9 +305,10 @@ int static_scratch(int device, void** out) {
       fc::set_cuda_error(e, "cudaGetSymbolAddress(g_decide_scratch)");
       return FC_ERR_CUDA;
     }
-    g_scratch_addr[device] = p;
+    g_scratch_addr[device].store(p, std::memory_order_release);
+    known = p;
   }
-  *out = g_scratch_addr[device];
+  *out = known;
   return FC_OK;
 }
 
@@ -271,8 +318,8 @@ extern "C" size_t fc_chunk_decide_static_max_bytes(void) { return kStaticScratch
 
 extern "C" int fc_chunk_decide_static(fc_ctx* ctx, void* stream, const void* cur, const void* prev, int dtype,
                                       const int64_t* chunk_elem_off, int n_chunks, const int32_t* chunk_step,
-                                      int warmup_m, float eps, const uint8_t* force, float* acc, float* l1rel,
-                                      uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
+                                      int warmup_m, float eps, const uint8_t* force, int policy, float* acc,
+                                      float* l1rel, uint8_t* recompute, int32_t* active_ids, int32_t* n_active,
                                       uint32_t* status) {
   if (!ctx || !chunk_elem_off || n_chunks <= 0) return FC_ERR_INVALID_ARG;
   if (n_chunks > FC_MAX_CHUNKS) return FC_ERR_UNSUPPORTED;
@@ -285,5 +332,5 @@ extern "C" int fc_chunk_decide_static(fc_ctx* ctx, void* stream, const void* cur
   // Every slab pair is written by the reduction before the finalising kernel reads it, so the
   // array needs no clearing between calls even though it keeps the previous call's contents.
   return fc_chunk_decide(ctx, stream, cur, prev, dtype, chunk_elem_off, n_chunks, chunk_step, warmup_m, eps, force,
-                         acc, l1rel, recompute, active_ids, n_active, status, scratch, kStaticScratchBytes);
+                         policy, acc, l1rel, recompute, active_ids, n_active, status, scratch, kStaticScratchBytes);
 }

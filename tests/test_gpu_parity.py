@@ -114,6 +114,89 @@ def test_decide_full_size(ctx, name):
     _run_decide_sequence(ctx, w.torch_dtype, lens, 2, 0.1, 1, w.seed)
 
 
+def test_decide_uniform_policy_sequence(ctx):
+    # the uniform policy (one shared decision; a re-initialised chunk is computed on its own) over ten steps,
+    # ragged chunk lengths, bit-exact flags against the oracle, no step inside the guard band of the threshold
+    from paper_2602_10825_b200 import binding
+    lens = [40000, 8192 * 3 + 8, 123456, 1001]
+    n, eps, m = len(lens), 0.12, 1
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    acc_o = np.zeros(n, np.float32)
+    acc_g = torch.zeros(n, device="cuda")
+    seen = set()
+    for s in range(10):
+        target = wl.uniform((n,), 770 + s, 0.0, 0.1)
+        parts = [wl.indicator_pair(1, int(L), [float(target[c])], 7700 + s * 10 + c) for c, L in enumerate(lens)]
+        cur, prev = torch.cat([p[0] for p in parts]), torch.cat([p[1] for p in parts])
+        step = np.full(n, s, np.int32)
+        if s >= 4:
+            step[2] = s - 4  # chunk 2 is re-initialised at step 4: in warm-up there, sharing again afterwards
+        force = np.array([0, 1 if s == 7 else 0, 0, 0], np.uint8)
+        want = oracle.chunk_decide_uniform(wl.bits(cur), wl.bits(prev), off, step, m, eps, acc_o, force=force)
+        sharing = (step >= m) & (force == 0)
+        if sharing.any():
+            first = int(np.flatnonzero(sharing)[0])
+            assert abs(acc_o[first] + want["l1rel"][first] - eps) > 1e-3 * eps, "inside the guard band: change the seed"
+        got = ctx.chunk_decide(dev(cur), dev(prev), off, i32(step), m, eps, acc_g, force=torch.from_numpy(force).cuda(),
+                               policy=binding.POLICY_UNIFORM)
+        torch.cuda.synchronize()
+        assert got["recompute"].cpu().numpy().tolist() == want["recompute"].tolist(), f"step {s}"
+        assert int(got["n_active"].item()) == want["n_active"]
+        ids = got["active_ids"].cpu().numpy()
+        assert ids[:want["n_active"]].tolist() == want["active_ids"].tolist() and (ids[want["n_active"]:] == -1).all()
+        np.testing.assert_allclose(got["l1rel"].cpu().numpy(), want["l1rel"], rtol=2e-6)
+        np.testing.assert_allclose(acc_g.cpu().numpy(), want["acc"], rtol=4e-6, atol=1e-9)
+        acc_o = want["acc"]
+        seen.add(tuple(want["recompute"].tolist()))
+    assert len(seen) >= 3  # all computed, all reused, and a mixed step around the re-initialised chunk
+
+
+# ------------------------------------------------------------------------------------ activation cache
+
+@pytest.mark.parametrize("dtype,lens", [(torch.bfloat16, [8192 * 3 + 8, 40000, 8, 123456]),  # 16-byte aligned offsets
+                                        (torch.bfloat16, [1001, 77777, 3]),                   # unaligned: scalar path
+                                        (torch.float32, [4100, 65536 + 4, 0, 12])])
+def test_cache_apply_bit_exact(ctx, dtype, lens):
+    # two steps: every chunk computed (the residuals are stored), then a mixed step (skipped chunks are served from
+    # the cache, computed ones refresh it); outputs and cache bit for bit against the oracle, untouched parts intact
+    n = len(lens)
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    E = int(off[-1])
+    cache_o = wl.bits(wl.normal((E,), 501, 1.0, dtype))
+    cache_g = dev(wl.normal((E,), 501, 1.0, dtype))
+    for s, rec in enumerate([[1] * n, [(c + 1) % 2 for c in range(n)], [0] * n]):
+        x = wl.normal((E,), 510 + s, 2.0, dtype)
+        y = wl.normal((E,), 520 + s, 2.0, dtype)
+        y_o, cache_o = oracle.chunk_cache_apply(wl.bits(x), wl.bits(y), cache_o, off, rec)
+        y_g = dev(y)
+        ctx.chunk_cache_apply(dev(x), y_g, cache_g, off, torch.tensor(rec, dtype=torch.uint8).cuda())
+        torch.cuda.synchronize()
+        assert np.array_equal(wl.bits(y_g.cpu()), y_o), f"step {s}"
+        assert np.array_equal(wl.bits(cache_g.cpu()), cache_o), f"step {s}"
+
+
+def test_cache_apply_full_size_follows_the_decision_on_the_device(ctx):
+    # config 3's indicator tensors (8 chunks x 4680 tokens x 3072): decide, then serve the skipped chunks, the flags
+    # going from one call to the other in device memory; every element against the oracle
+    w = wl.CONFIGS["cached_step_bf16"]
+    n_el = w.n_c * w.hidden
+    off = np.arange(w.W + 1, dtype=np.int64) * n_el
+    target = [0.3, 0.01, 0.3, 0.02, 0.01, 0.3, 0.02, 0.3]
+    cur, prev = wl.indicator_pair(w.W, n_el, target, 4)
+    step = np.full(w.W, 6, np.int32)
+    want_d = oracle.chunk_decide(wl.bits(cur), wl.bits(prev), off, step, 1, 0.1, np.zeros(w.W, np.float32))
+    dec = ctx.chunk_decide(dev(cur), dev(prev), off, i32(step), 1, 0.1, torch.zeros(w.W, device="cuda"))
+    y = wl.normal((w.W * n_el,), 44, 1.0, torch.bfloat16)
+    cache = wl.normal((w.W * n_el,), 45, 0.1, torch.bfloat16)
+    y_g, cache_g = dev(y), dev(cache)
+    ctx.chunk_cache_apply(dev(cur), y_g, cache_g, off, dec["recompute"])
+    torch.cuda.synchronize()
+    assert dec["recompute"].cpu().numpy().tolist() == want_d["recompute"].tolist() == [1, 0, 1, 0, 0, 1, 0, 1]
+    y_o, cache_o = oracle.chunk_cache_apply(wl.bits(cur), wl.bits(y), wl.bits(cache), off, want_d["recompute"])
+    assert np.array_equal(wl.bits(y_g.cpu()), y_o)
+    assert np.array_equal(wl.bits(cache_g.cpu()), cache_o)
+
+
 # ------------------------------------------------------------------------------------ attention
 
 def _attention_case(ctx, w, active, *, impl=0, token_map=False, sample=None, atol, rel_l2, check_lse=True):
@@ -145,14 +228,15 @@ def _attention_case(ctx, w, active, *, impl=0, token_map=False, sample=None, ato
         wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, None if token_map else slo,
         None if token_map else spo, active, kv_token_index=tok, sample_rows=sample,
         O_init=None if sample is not None else O0.double().numpy())
-    got = Og.double().cpu().numpy()
-    lse_got = lse_g.double().cpu().numpy()
     if sample is not None:
         rows = np.asarray(sample)
         is_act = np.isin(rows // w.n_c, list(active))
-        got_s, want_s = got[:, rows[is_act]], O_want[:, is_act]
-        lse_got_s, lse_want_s = lse_got[:, rows[is_act]], lse_want[:, is_act]
+        pick = torch.as_tensor(rows[is_act], dtype=torch.long, device="cuda")  # gathered on the device: O is large
+        got_s, want_s = Og[:, pick].double().cpu().numpy(), O_want[:, is_act]
+        lse_got_s, lse_want_s = lse_g[:, pick].double().cpu().numpy(), lse_want[:, is_act]
     else:
+        got = Og.double().cpu().numpy()
+        lse_got = lse_g.double().cpu().numpy()
         rows_act = np.concatenate([np.arange(q_off[c], q_off[c + 1]) for c in active]) if active else np.array([], int)
         got_s, want_s = got[:, rows_act], O_want[:, rows_act]
         lse_got_s, lse_want_s = lse_got[:, rows_act], lse_want[:, rows_act]
@@ -195,9 +279,8 @@ def test_attention_token_index_map(ctx):
     _attention_case(ctx, wb, [1], token_map=True, atol=1e-2, rel_l2=1e-2)
 
 
-@pytest.mark.parametrize("impl", [2, 3])  # warp-specialised and single-stage tcgen05 kernels
 @pytest.mark.parametrize("d", [128, 64])
-def test_attention_bf16_tensor_core_small(ctx, impl, d):
+def test_attention_bf16_tensor_core_small(ctx, d, impl=2):
     # several 128-row tiles with ragged tails in both rows and keys, a clean region and a window
     w = wl.Workload("t", "bf16", H=2, d=d, W=3, n_c=328, B=200, L_k=528, seed=15, sigma=0.5)
     _attention_case(ctx, w, [0, 1, 2], impl=impl, atol=1e-2, rel_l2=1e-2)
@@ -230,8 +313,7 @@ def _attention_custom(ctx, Q, K, V, q_off, vis, slo, spo, active, impl, O0=None)
     return Og
 
 
-@pytest.mark.parametrize("impl", [2, 3])
-def test_attention_tensor_core_edge_cases(ctx, impl):
+def test_attention_tensor_core_edge_cases(ctx, impl=2):
     d = 128
     # grouped query heads: 4 query heads on 2 key heads
     Q = wl.normal((4, 300, d), 61, 0.5, torch.bfloat16)
@@ -264,17 +346,92 @@ def test_attention_tensor_core_edge_cases(ctx, impl):
     assert torch.equal(Og.cpu(), O0)
 
 
+def _poison_unreferenced_rows(K, V, vis_max, slo, spo):
+    """Overwrite every physical K/V row that no visible logical token maps to with NaN, +-inf and +-3e38."""
+    L = K.shape[1]
+    used = np.zeros(L, bool)
+    for s_ in range(len(spo)):
+        n = min(int(slo[s_ + 1]), vis_max) - int(slo[s_])
+        if n > 0:
+            used[int(spo[s_]):int(spo[s_]) + n] = True
+    bad = torch.tensor([float("nan"), float("inf"), -float("inf"), 3e38, -3e38], dtype=torch.float32)
+    rows = np.flatnonzero(~used)
+    fill = bad[torch.arange(len(rows)) % 5].to(torch.bfloat16)[None, :, None]
+    K[:, rows] = fill
+    V[:, rows] = fill.flip(1)
+    return len(rows)
+
+
+@pytest.mark.parametrize("d", [128, 64])
+def test_attention_ignores_rows_outside_the_visible_segments(ctx, d):
+    # The K/V buffer of the method has slots that are not written yet, and a segment's last 128-row tile drags in
+    # whatever follows the segment.  Every such row is filled with NaN, infinities and 3e38 here: the outputs must
+    # still match the oracle (which never reads those rows) and be finite.
+    rng = np.random.default_rng(4)
+    # (1) a clean region scattered over segments with gaps, as in the edge-case test
+    seg_len = [37, 128, 1, 255, 64, 129, 90, 7, 300, 13]
+    order = rng.permutation(len(seg_len))
+    phys = np.zeros(len(seg_len), np.int64)
+    pos = 5
+    for s_ in order:
+        phys[s_] = pos
+        pos += seg_len[s_] + int(rng.integers(1, 9))
+    slo = np.concatenate([[0], np.cumsum(seg_len)]).astype(np.int32)
+    L_phys = pos + 130
+    Q = wl.normal((2, 700, d), 64, 0.5, torch.bfloat16)
+    K = wl.normal((2, L_phys, d), 65, 0.5, torch.bfloat16)
+    V = wl.normal((2, L_phys, d), 66, 0.5, torch.bfloat16)
+    q_off = np.array([0, 130, 400, 700], np.int32)
+    vis = np.array([slo[-1], 700, 166], np.int32)
+    assert _poison_unreferenced_rows(K, V, int(slo[-1]), slo, phys) > 100
+    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, phys.astype(np.int32), [0, 1, 2], 2)
+    assert torch.isfinite(Og.float()).all()
+    # (2) the prefix layout [clean region | gap | chunk 0 | gap | chunk 1 | unwritten rest], the second chunk's slot
+    # only partly written: chunk 1 sees 100 of its 328 rows, the other 228 are poison inside its own segment
+    B, n_c = 200, 328
+    spo = np.array([0, B + 56, B + 56 + n_c + 100], np.int32)
+    slo = np.array([0, B, B + n_c, B + 2 * n_c], np.int32)
+    L_phys = int(spo[2]) + n_c + 77
+    Q = wl.normal((3, 2 * n_c, d), 67, 0.5, torch.bfloat16)
+    K = wl.normal((3, L_phys, d), 68, 0.5, torch.bfloat16)
+    V = wl.normal((3, L_phys, d), 69, 0.5, torch.bfloat16)
+    q_off = np.array([0, n_c, 2 * n_c], np.int32)
+    vis = np.array([B + n_c, B + n_c + 100], np.int32)
+    assert _poison_unreferenced_rows(K, V, int(vis[1]), slo, spo) > 400
+    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, spo, [0, 1], 2)
+    assert torch.isfinite(Og.float()).all()
+    # the CUDA-core kernel reads through the same tables
+    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, spo, [0, 1], 1)
+    assert torch.isfinite(Og.float()).all()
+
+
 def test_attention_bf16_many_items_per_cta(ctx):
     # more work items than SMs, of very different lengths: exercises the device-side item queue
     w = wl.Workload("q", "bf16", H=40, d=128, W=6, n_c=520, B=300, L_k=820, seed=18, sigma=0.5)
     _attention_case(ctx, w, [0, 1, 3, 5], impl=2, sample=wl.sample_rows(w, 40, 1), atol=1e-2, rel_l2=1e-2)
 
 
-@pytest.mark.parametrize("name,active", [("single_step_bf16", [0, 1, 2, 3]), ("cached_step_bf16", [2, 5, 7])])
-def test_attention_full_size_sampled_rows(ctx, name, active):
-    # the launch configuration the benchmark times, checked on sampled query rows over the full key range
+# The launch configurations the benchmark times, at full size, on sampled query rows over the full key range:
+# boundary rows of every active chunk plus uniform draws from the active chunks (4096 on the single-step
+# configuration, 1024 on the others; the sparse sweep list and the second model family take 512).
+FULL_SIZE_CASES = [
+    ("single_step_bf16", [0, 1, 2, 3], 4096),
+    ("cached_step_bf16", [2, 5, 7], 1024),
+    ("streaming_bf16", [0], 1024),                 # one chunk over the 28080-token history
+    ("sweep_bf16", list(range(16)), 1024),         # every chunk of the window recomputed
+    ("sweep_bf16", [1, 4, 9, 15], 512),            # a sparse active list late in the sweep
+    ("skyreels_bf16", [0, 2, 3], 512),
+]
+
+
+@pytest.mark.parametrize("name,active,n_uniform", FULL_SIZE_CASES,
+                         ids=[f"{n}-{len(a)}of{wl.CONFIGS[n].W}" for n, a, _ in FULL_SIZE_CASES])
+def test_attention_full_size_sampled_rows(ctx, name, active, n_uniform):
     w = wl.CONFIGS[name]
-    _attention_case(ctx, w, active, sample=wl.sample_rows(w, 48, 2), atol=1e-2, rel_l2=1e-2)
+    rows = wl.sample_rows(w, n_uniform, 2, chunks=active)
+    assert len(rows) >= n_uniform * 0.9
+    _attention_case(ctx, w, active, sample=rows, atol=1e-2, rel_l2=1e-2)
+    torch.cuda.empty_cache()
 
 
 def test_attention_bf16_matches_cuda_core_kernel(ctx):
@@ -524,6 +681,12 @@ def test_bad_arguments_return_a_status_and_launch_nothing(ctx):
         ctx.chunk_attention(Qm, K, V, q_off, vis, slo, spo, act, n_act, O)
     with pytest.raises(fc.FcError, match="invalid"):
         ctx.kv_score(Q[:, :50], K, pool_k=4)
+    with pytest.raises(fc.FcError, match="invalid"):  # the cache must be a tensor of its own
+        flat = Q.view(-1)
+        ctx.chunk_cache_apply(flat, flat.clone(), flat, [0, flat.numel()], torch.zeros(1, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(fc.FcError, match="invalid"):
+        ctx.chunk_decide(Q.view(-1), K.view(-1)[:Q.numel()], [0, Q.numel()], i32([0]), 1, 0.1,
+                         torch.zeros(1, device="cuda"), policy=7)
     with pytest.raises(fc.FcError, match="invalid"):
         bad_vis = vis.copy()
         bad_vis[-1] += 1  # beyond the logical length

@@ -195,3 +195,94 @@ def test_blocks_at_staggered_noise_levels(ctx, eps):
                 if c not in active:
                     assert torch.equal(O[:, q_off[c]:q_off[c + 1]].cpu(), O0[:, q_off[c]:q_off[c + 1]])
     assert n_forced > 0 and n_reused > 0
+
+
+# ------------------------------------------------------------------------------------ full-size compression events
+
+def _guarded(H, n_keep, d, dtype):
+    """A destination [H, n_keep, d] with one canary row before and one after every head's rows."""
+    buf = torch.full((H, n_keep + 2, d), 7.0, dtype=dtype, device="cuda")
+    return buf, buf[:, 1:n_keep + 1]
+
+
+@pytest.mark.parametrize("name", ["cached_step_bf16", "streaming_bf16", "sweep_bf16"])
+def test_compression_event_at_full_size_every_element(ctx, name):
+    # One compression event of the configuration exactly as the benchmark launches it (all heads, L_k candidates,
+    # budget B): the scores against the oracle on every element; the selection on the library's own fp32 scores
+    # fed to both sides, indices bit-exact; the compacted K and V rows byte-exact; canary rows before and after
+    # every destination head untouched.
+    w = wl.CONFIGS[name]
+    Q_obs, K, V = wl.candidates(w)
+    Kg, Vg = K.cuda(), V.cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    imp = torch.empty((w.H, w.L_k), device="cuda")
+    red = torch.empty((w.H, w.L_k), device="cuda")
+    got = ctx.kv_score(Q_obs.cuda(), Kg, lambda_=w.lam, pool_k=w.pool_k, imp=imp, red=red, status=status)
+    K_buf, K_dst = _guarded(w.H, w.B, w.d, K.dtype)
+    V_buf, V_dst = _guarded(w.H, w.B, w.d, K.dtype)
+    sel = ctx.kv_select_compact(got["score"], w.B, Kg, Vg, K_dst, V_dst, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    want = oracle.kv_score(wl.bits(Q_obs), wl.bits(K), lambda_=w.lam, pool_k=w.pool_k)
+    for nm, g_, w_ in (("imp", imp, want["imp"]), ("red", red, want["red"]),
+                       ("score", got["score"], want["score"].astype(np.float64))):
+        g_ = g_.double().cpu().numpy()
+        assert (np.abs(g_ - w_) <= 1e-4 * np.abs(w_).max(axis=1, keepdims=True)).all(), nm
+    score = got["score"].cpu().numpy()
+    want_sel = oracle.kv_select_compact(score, w.B, wl.bits(K), wl.bits(V))
+    assert int(sel["n_kept"].item()) == want_sel["n_kept"] == w.B
+    assert np.array_equal(sel["kept_idx"].cpu().numpy(), want_sel["kept_idx"])
+    assert np.array_equal(wl.bits(K_dst.cpu()), want_sel["K_dst"])
+    assert np.array_equal(wl.bits(V_dst.cpu()), want_sel["V_dst"])
+    for buf in (K_buf, V_buf):
+        assert (buf[:, 0] == 7.0).all() and (buf[:, w.B + 1] == 7.0).all()
+
+
+def test_streaming_generation_at_full_width(ctx):
+    # config 4 at full width (24 heads, chunks of 4680 tokens, budget 28080): the history starts full, then eight
+    # chunks are generated one after another, each with S denoising steps of attention over [history | itself]
+    # (sampled rows) and an accumulated importance, and a real compression 32760 -> 28080 after every chunk,
+    # selection bit-exact on the library's scores and rows byte-exact, every time.
+    full = wl.CONFIGS["streaming_bf16"]
+    H, d, n_c, B, S = full.H, full.d, full.n_c, full.B, full.n_steps
+    n_chunks, n_fill = 8, full.B // full.n_c
+    keys = list(wl.ar1_keys(H, n_fill + n_chunks, n_c, d, seed=full.seed, sigma=full.sigma))
+    hist_K = torch.cat(keys[:n_fill], 1).contiguous()
+    hist_V = wl.normal((H, B, d), 6999, full.sigma, torch.bfloat16)
+    q_off, vis = np.array([0, n_c], np.int32), np.array([B + n_c], np.int32)
+    slo, spo = np.array([0, B, B + n_c], np.int32), np.array([0, B], np.int32)
+    shape = wl.Workload("x", "bf16", H=H, d=d, W=1, n_c=n_c, B=0, L_k=0, seed=0)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for c in range(n_chunks):
+        K_all = torch.cat([hist_K, keys[n_fill + c]], 1).contiguous()
+        V_all = torch.cat([hist_V, wl.normal((H, n_c, d), 7000 + c, full.sigma, torch.bfloat16)], 1).contiguous()
+        Kg, Vg = K_all.cuda(), V_all.cuda()
+        acc_g = torch.zeros((H, B + n_c), device="cuda")
+        acc_o = np.zeros((H, B + n_c), np.float64)
+        for s in range(S):
+            Q = wl.normal((H, n_c, d), 8000 + 10 * c + s, full.sigma, torch.bfloat16)
+            O = torch.zeros((H, n_c, d), dtype=torch.bfloat16, device="cuda")
+            ctx.chunk_attention(Q.cuda(), Kg, Vg, q_off, vis, slo, spo, i32([0]), i32([1]), O, status=status)
+            rows = wl.sample_rows(shape, 8, 10 * c + s)
+            O_want, _ = oracle.chunk_attention(wl.bits(Q), wl.bits(K_all), wl.bits(V_all), q_off, vis, slo, spo, [0],
+                                               sample_rows=rows)
+            _check_attention(O[:, torch.as_tensor(rows, dtype=torch.long, device="cuda")].double().cpu().numpy(), O_want)
+            Q_obs = Q[:, n_c - full.L_q_obs:].contiguous()
+            phase = 2 if s == S - 1 else 1
+            want = oracle.kv_score(wl.bits(Q_obs), wl.bits(K_all), lambda_=full.lam, pool_k=full.pool_k,
+                                   imp_accum=acc_o, accum_phase=phase, n_steps=S)
+            got = ctx.kv_score(Q_obs.cuda(), Kg, lambda_=full.lam, pool_k=full.pool_k, imp_accum=acc_g,
+                               accum_phase=phase, n_steps=S, status=status)
+        torch.cuda.synchronize()
+        score = got["score"].cpu().numpy()
+        assert np.abs(score - want["score"]).max() <= 1e-4 * np.abs(want["score"]).max()
+        sel = ctx.kv_select_compact(got["score"], B, Kg, Vg, status=status)
+        want_sel = oracle.kv_select_compact(score, B, wl.bits(K_all), wl.bits(V_all))
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        assert sel["kept_idx"].shape == (H, B)
+        assert np.array_equal(sel["kept_idx"].cpu().numpy(), want_sel["kept_idx"])
+        assert np.array_equal(wl.bits(sel["K_dst"].cpu()), want_sel["K_dst"])
+        assert np.array_equal(wl.bits(sel["V_dst"].cpu()), want_sel["V_dst"])
+        assert not np.array_equal(want_sel["kept_idx"][0], np.arange(B, dtype=np.int32))  # something was dropped
+        hist_K, hist_V = sel["K_dst"].cpu(), sel["V_dst"].cpu()

@@ -1,17 +1,19 @@
-"""The no-allocation entry point fc_chunk_decide_static against fc_chunk_decide.
+"""The no-allocation entry point fc_chunk_decide_static against fc_chunk_decide and against the CPU oracle.
 
 Some callers cannot allocate device memory where they call the library (inside an allocator or
 memory-pool callback, in a loop that must stay off the allocator, or when another runtime owns all
 device memory and hands out fixed buffers), so they have no workspace to give.  For them the
 decision kernel has a twin whose scratch is a fixed 1 MiB array inside the library.  This test
 calls the twin through the C ABI twice in a row (the array keeps the first call's contents) and
-checks both results against the workspace-taking entry point on the same inputs.  It is collected
-last so that a run stopping at the first failure has already run every other test.
+checks both results against the workspace-taking entry point on the same inputs, and first-hand
+against the oracle's statement of Eqs. 5 and 8.  It is collected last so that a run stopping at the
+first failure has already run every other test.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -34,8 +36,8 @@ def test_static_scratch_decide_matches_workspace_decide_twice():
              ([4096 * 7, 999], [0.3, 0.01], torch.float32, 0.1, 12)]
     for lens, target, dtype, eps, seed in cases:
         parts = [wl.indicator_pair(1, L, [r], seed * 10 + i, dtype=dtype) for i, (L, r) in enumerate(zip(lens, target))]
-        cur = torch.cat([p[0] for p in parts]).cuda()
-        prev = torch.cat([p[1] for p in parts]).cuda()
+        cur_h, prev_h = torch.cat([p[0] for p in parts]), torch.cat([p[1] for p in parts])
+        cur, prev = cur_h.cuda(), prev_h.cuda()
         off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
         n = len(lens)
         step = torch.full((n,), 3, dtype=torch.int32, device="cuda")
@@ -52,6 +54,15 @@ def test_static_scratch_decide_matches_workspace_decide_twice():
         np.testing.assert_allclose(new["l1rel"].cpu().numpy(), ref["l1rel"].cpu().numpy(), rtol=2e-6)
         np.testing.assert_allclose(acc_new.cpu().numpy(), acc_ref.cpu().numpy(), rtol=4e-6, atol=1e-9)
         assert int(ref["n_active"].item()) >= 1
+        # and against the oracle itself: decisions bit-exact, no chunk within the guard band of the threshold
+        want = oracle.chunk_decide(wl.bits(cur_h), wl.bits(prev_h), off, np.full(n, 3, np.int32), 1, eps,
+                                   acc0.cpu().numpy())
+        assert np.abs(acc0.cpu().numpy() + want["l1rel"] - eps).min() > 1e-3 * eps
+        assert new["recompute"].cpu().numpy().tolist() == want["recompute"].tolist()
+        assert int(new["n_active"].item()) == want["n_active"]
+        assert new["active_ids"].cpu().numpy()[:want["n_active"]].tolist() == want["active_ids"].tolist()
+        np.testing.assert_allclose(new["l1rel"].cpu().numpy(), want["l1rel"], rtol=2e-6)
+        np.testing.assert_allclose(acc_new.cpu().numpy(), want["acc"], rtol=4e-6, atol=1e-9)
     # a problem whose slab pairs would not fit the array is refused, and nothing is launched
     big = 300_000_000
     out = _outputs(1)

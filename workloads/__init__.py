@@ -185,18 +185,24 @@ def sweep_targets(n_steps, n_chunks, seed, kappa_end=0.02):
     return u * kappa[:, None]
 
 
-def sample_rows(w: Workload, n_uniform, seed, tile=128):
+def sample_rows(w: Workload, n_uniform, seed, tile=128, chunks=None):
     """Query rows for sampled parity: first / last row of every chunk, the rows on either side of
-    every ``tile`` boundary class (first tile, last full tile, ragged tail), plus uniform draws."""
+    every ``tile`` boundary class (first tile, last full tile, ragged tail), plus ``n_uniform`` distinct
+    rows drawn uniformly.  With ``chunks`` (a list of chunk ids) both kinds come from those chunks only."""
+    chunks = list(range(w.W)) if chunks is None else [int(c) for c in chunks]
     rows = set()
-    for c in range(w.W):
+    for c in chunks:
         base = c * w.n_c
         last_full = (w.n_c // tile) * tile
         for r in (0, 1, tile - 1, tile, last_full - 1, last_full, w.n_c - 2, w.n_c - 1):
             if 0 <= r < w.n_c:
                 rows.add(base + r)
-    extra = torch.randint(0, w.window_rows, (n_uniform,), generator=_gen(w.seed * 1000 + 900 + seed))
-    rows.update(int(x) for x in extra)
+    if chunks and n_uniform > 0:
+        # distinct rows: a random permutation of the chunks' rows, cut to n_uniform
+        pool = len(chunks) * w.n_c
+        pick = torch.randperm(pool, generator=_gen(w.seed * 1000 + 900 + seed))[:n_uniform]
+        extra = torch.tensor(chunks)[pick // w.n_c] * w.n_c + pick % w.n_c
+        rows.update(int(x) for x in extra)
     return np.asarray(sorted(rows), np.int32)
 
 

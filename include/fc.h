@@ -236,6 +236,16 @@ int fc_chunk_attention(fc_ctx* ctx, void* stream, const fc_attn_desc* desc, cons
  * to 8192 - take the frame-level pipeline, in which both passes over the logits run on the
  * tensor cores.
  */
+/* How the softmax argument of the redundancy (Eq. 11) is evaluated.
+ *   FC_RED_MEANKEY    the mean-key identity of the efficiency appendix (default; O(L_k d) per head)
+ *   FC_RED_TILED      Eq. 11 as written: 128 x 128 tiles of the cosine matrix on the tensor cores, diagonal
+ *                     zeroed, column sums in the epilogue, the matrix never stored (O(L_k^2 d) per head: the
+ *                     dense work the identity avoids; for checking it and as the base of the next mode)
+ *   FC_RED_TILED_MAX  not in the paper: the column MAXIMUM over the other tokens instead of the column mean,
+ *                     a statistic no mean key can express (same tiles, another epilogue)
+ * The tiled modes need bf16 keys. */
+typedef enum { FC_RED_MEANKEY = 0, FC_RED_TILED = 1, FC_RED_TILED_MAX = 2 } fc_red_mode;
+
 typedef struct {
   int32_t H_q, H_kv, d, L_q, L_k;  /* L_q * (H_q/H_kv) <= 128, or bf16 with H_q == H_kv and L_q <= 8192 */
   int64_t q_hs, q_rs, k_hs, k_rs;  /* element strides */
@@ -243,6 +253,7 @@ typedef struct {
   float lambda;                    /* mixing coefficient (paper: 0.07) */
   int32_t pool_k;                  /* odd, >= 1 */
   int32_t impl;                    /* 0 auto; 1 force the CUDA-core kernels; 2 force tcgen05 */
+  int32_t red_mode;                /* fc_red_mode */
 } fc_score_desc;
 
 /*   Q_obs            DEVICE [H_q, L_q, d]; K_cand DEVICE [H_kv, L_k, d]; `dtype` elements.

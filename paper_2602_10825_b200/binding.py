@@ -15,6 +15,7 @@ _HEADER = os.path.join(_ROOT, "include", "fc.h")
 
 BF16, F32 = 0, 1
 POLICY_CHUNKWISE, POLICY_UNIFORM = 0, 1
+RED_MEANKEY, RED_TILED, RED_TILED_MAX = 0, 1, 2
 STATUS_BITS = {"timeout": 1, "nan_score": 2, "bad_index": 4}
 
 
@@ -33,7 +34,7 @@ class _ScoreDesc(C.Structure):
     _fields_ = [("H_q", C.c_int32), ("H_kv", C.c_int32), ("d", C.c_int32), ("L_q", C.c_int32),
                 ("L_k", C.c_int32), ("q_hs", C.c_int64), ("q_rs", C.c_int64), ("k_hs", C.c_int64),
                 ("k_rs", C.c_int64), ("scale", C.c_float), ("lambda_", C.c_float),
-                ("pool_k", C.c_int32), ("impl", C.c_int32)]
+                ("pool_k", C.c_int32), ("impl", C.c_int32), ("red_mode", C.c_int32)]
 
 
 class _CompactStrides(C.Structure):
@@ -248,12 +249,12 @@ class Context:
 
     # ------------------------------------------------------------------ fc_kv_score
     def kv_score(self, Q_obs, K_cand, *, lambda_=0.07, pool_k=7, scale=0.0, imp_accum=None, accum_phase=0,
-                 n_steps=1, imp=None, red=None, score=None, impl=0, status=None, ws=None):
+                 n_steps=1, imp=None, red=None, score=None, impl=0, red_mode=RED_MEANKEY, status=None, ws=None):
         q_hs, q_rs = _hsr(Q_obs, "Q_obs")
         k_hs, k_rs = _hsr(K_cand, "K_cand")
         H_kv, L_k, d = K_cand.shape
         desc = _ScoreDesc(Q_obs.shape[0], H_kv, d, Q_obs.shape[1], L_k, q_hs, q_rs, k_hs, k_rs, scale, lambda_,
-                          pool_k, impl)
+                          pool_k, impl, red_mode)
         if score is None and accum_phase != 1:
             score = torch.empty((H_kv, L_k), dtype=torch.float32, device=K_cand.device)
         for name, t in (("imp", imp), ("red", red), ("score", score), ("imp_accum", imp_accum)):

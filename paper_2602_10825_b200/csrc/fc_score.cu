@@ -273,6 +273,7 @@ struct ScoreWs {
   float* tc_lse2;
   float* tc_norm2;
   // frame-level path
+  float* inv_norm;     // tiled redundancy: [H, n_tiles * 128] reciprocal key norms
   float* fr_mass;      // [H, L_k] sum over the queries of exp(logit - lse)
   float2* fr_ml;       // [H, slices, L_q] (maximum, sum) of every query over a slice of the keys
   size_t total;
@@ -298,6 +299,7 @@ ScoreWs carve(const ScoreGeom& g, void* ws) {
   w.tc_colsum = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxSlices * g.d * 4);
   w.tc_lse2 = (float*)take((size_t)g.H_kv * fc::kScoreTcMaxQueries * 4);
   w.tc_norm2 = (float*)take((size_t)g.H_kv * g.L_k * 4);
+  w.inv_norm = (float*)take((size_t)g.H_kv * g.n_tiles * kTile * 4);
   w.fr_mass = (float*)take(frame ? (size_t)g.H_kv * g.L_k * 4 : 0);
   w.fr_ml = (float2*)take(frame ? (size_t)g.H_kv * fc::kScoreFrameMaxSlices * g.L_q * 8 : 0);
   w.total = off;
@@ -324,7 +326,7 @@ int make_geom(const fc_score_desc* d, ScoreGeom& g) {
 
 template <typename T, int D>
 int run(cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, const void* K,
-        float* imp_accum, int phase, int n_steps, float* imp, float* red, float* score) {
+        float* imp_accum, int phase, int n_steps, float* imp_buf) {
   const size_t smem1 = ((size_t)g.n_q * D + (size_t)kTile * (D + 1)) * 4;
   FC_CUDA_CHECK(cudaFuncSetAttribute(score_pass1_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)smem1));
@@ -335,21 +337,16 @@ int run(cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, co
   FC_LAUNCH_CHECK("score_row_lse_kernel");
   score_mean_key_kernel<<<g.H_kv, 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
   FC_LAUNCH_CHECK("score_mean_key_kernel");
-  float* imp_buf = imp ? imp : w.imp_tmp;
   score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, w.S, w.lse, w.mean_key, nullptr, imp_accum, phase,
                                                    n_steps, imp_buf, w.a, w.a_partial);
   FC_LAUNCH_CHECK("score_pass2_kernel");
-  if (phase != 1) {
-    score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
-    FC_LAUNCH_CHECK("score_finalize_kernel");
-  }
   return FC_OK;
 }
 
 // Frame-level pipeline (bf16, one query head per key head, any number of queries up to kScoreFrameMaxQueries).
 template <int D>
 int run_frame(fc_ctx* ctx, cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, const void* K,
-              float* imp_accum, int phase, int n_steps, float* imp, float* red, float* score, uint32_t* status) {
+              float* imp_accum, int phase, int n_steps, float* imp_buf, uint32_t* status) {
   using T = __nv_bfloat16;
   dim3 grid(g.n_tiles, g.H_kv);
   // 1. sums of normalised keys per tile (no queries: the logit loop of the kernel is empty)
@@ -365,15 +362,10 @@ int run_frame(fc_ctx* ctx, cudaStream_t st, const ScoreGeom& g, const ScoreWs& w
   int rc = fc::score_frame_mass(ctx, st, g.H_kv, g.d, g.L_q, g.L_k, g.scale * 1.4426950408889634f, Q, g.q_hs, g.q_rs, K,
                                 g.k_hs, g.k_rs, w.fr_ml, w.lse, w.fr_mass, status);
   if (rc != FC_OK) return rc;
-  // 4. mean over the queries, accumulation over steps, redundancy logits; 5. finalize
-  float* imp_buf = imp ? imp : w.imp_tmp;
+  // 4. mean over the queries, accumulation over steps, redundancy logits
   score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, nullptr, nullptr, w.mean_key, w.fr_mass, imp_accum,
                                                    phase, n_steps, imp_buf, w.a, w.a_partial);
   FC_LAUNCH_CHECK("score_pass2_kernel");
-  if (phase != 1) {
-    score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
-    FC_LAUNCH_CHECK("score_finalize_kernel");
-  }
   return FC_OK;
 }
 
@@ -407,32 +399,47 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
   if (!fc::aligned16(ws)) return FC_ERR_MISALIGNED;
   cudaStream_t st = (cudaStream_t)stream;
   if (desc->impl < 0 || desc->impl > 2) return FC_ERR_INVALID_ARG;
+  if (desc->red_mode < FC_RED_MEANKEY || desc->red_mode > FC_RED_TILED_MAX) return FC_ERR_INVALID_ARG;
+  if (desc->red_mode != FC_RED_MEANKEY && dtype != FC_BF16) return FC_ERR_UNSUPPORTED;  // the tiles are bf16 MMAs
+  float* imp_buf = imp ? imp : w.imp_tmp;
+  // 1. importance (and the mean-key redundancy argument) by one of the three pipelines
   if (g.n_q > kCoreMaxQueries) {
     if (dtype != FC_BF16 || desc->impl == 1) return FC_ERR_UNSUPPORTED;
-    if (g.d == 128) return run_frame<128>(ctx, st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score, status);
-    return run_frame<64>(ctx, st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score, status);
+    rc = g.d == 128 ? run_frame<128>(ctx, st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp_buf, status)
+                    : run_frame<64>(ctx, st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp_buf, status);
+  } else {
+    const bool tc_ok = dtype == FC_BF16 && g.group == 1 && g.L_q <= fc::kScoreTcMaxQueries - 2;
+    if (desc->impl == 2 && !tc_ok) return FC_ERR_UNSUPPORTED;
+    if (tc_ok && desc->impl != 1) {
+      fc::ScoreTcArgs a;
+      a.H = g.H_kv; a.L_q = g.L_q; a.L_k = g.L_k; a.n_tiles = g.n_tiles; a.tiles_per_slice = 0; a.n_slices = 0;
+      a.scale_log2 = g.scale * 1.4426950408889634f;
+      a.accum_phase = accum_phase; a.n_steps = n_steps;
+      a.ml_part = w.tc_ml; a.colsum_part = w.tc_colsum; a.norm2 = w.tc_norm2;
+      a.imp_accum = imp_accum; a.imp_out = imp_buf; a.a_out = w.a; a.a_partial = w.a_partial;
+      a.status = status;
+      rc = fc::score_tc_run(ctx, st, a, g.d, g.q_hs, g.q_rs, g.k_hs, g.k_rs, Q_obs, K_cand);
+      g.n_partials = g.n_tiles * 4;  // the tensor-core pass leaves one entry per warp of a tile
+    } else if (dtype == FC_BF16) {
+      rc = g.d == 128 ? run<__nv_bfloat16, 128>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp_buf)
+                      : run<__nv_bfloat16, 64>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp_buf);
+    } else {
+      rc = g.d == 128 ? run<float, 128>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp_buf)
+                      : run<float, 64>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp_buf);
+    }
   }
-  const bool tc_ok = dtype == FC_BF16 && g.group == 1 && g.L_q <= fc::kScoreTcMaxQueries - 2;
-  if (desc->impl == 2 && !tc_ok) return FC_ERR_UNSUPPORTED;
-  if (tc_ok && desc->impl != 1) {
-    fc::ScoreTcArgs a;
-    a.H = g.H_kv; a.L_q = g.L_q; a.L_k = g.L_k; a.n_tiles = g.n_tiles; a.tiles_per_slice = 0; a.n_slices = 0;
-    a.scale_log2 = g.scale * 1.4426950408889634f;
-    a.accum_phase = accum_phase; a.n_steps = n_steps;
-    a.ml_part = w.tc_ml; a.colsum_part = w.tc_colsum; a.norm2 = w.tc_norm2;
-    a.imp_accum = imp_accum; a.imp_out = imp ? imp : w.imp_tmp; a.a_out = w.a; a.a_partial = w.a_partial;
-    a.status = status;
-    rc = fc::score_tc_run(ctx, st, a, g.d, g.q_hs, g.q_rs, g.k_hs, g.k_rs, Q_obs, K_cand);
-    if (rc != FC_OK || accum_phase == 1) return rc;
-    g.n_partials = g.n_tiles * 4;  // the tensor-core pass leaves one entry per warp of a tile
-    score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, a.imp_out, w.a, w.a_partial, red, score);
-    FC_LAUNCH_CHECK("score_finalize_kernel");
-    return FC_OK;
+  if (rc != FC_OK || accum_phase == 1) return rc;
+  // 2. optionally the redundancy argument from explicit similarity tiles, in place of the mean-key form
+  if (desc->red_mode != FC_RED_MEANKEY) {
+    fc::RedTiledArgs r;
+    r.H = g.H_kv; r.L_k = g.L_k; r.n_tiles = g.n_tiles;
+    r.inv_norm = w.inv_norm; r.a_out = w.a; r.a_partial = w.a_partial; r.status = status;
+    rc = fc::score_red_tiled(ctx, st, r, g.d, g.k_hs, g.k_rs, K_cand, desc->red_mode == FC_RED_TILED_MAX);
+    if (rc != FC_OK) return rc;
+    g.n_partials = g.n_tiles * 4;
   }
-  if (dtype == FC_BF16) {
-    if (g.d == 128) return run<__nv_bfloat16, 128>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
-    return run<__nv_bfloat16, 64>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
-  }
-  if (g.d == 128) return run<float, 128>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
-  return run<float, 64>(st, g, w, Q_obs, K_cand, imp_accum, accum_phase, n_steps, imp, red, score);
+  // 3. softmax of the redundancy argument, max-pool of the importance, lambda-mix
+  score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
+  FC_LAUNCH_CHECK("score_finalize_kernel");
+  return FC_OK;
 }

@@ -31,6 +31,19 @@ struct ScoreTcArgs {
 int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs args, int d, int64_t q_hs, int64_t q_rs, int64_t k_hs,
                  int64_t k_rs, const void* Q, const void* K);
 
+// Redundancy from explicit tiles of the cosine-similarity matrix (fc_score_red.cu).
+struct RedTiledArgs {
+  int H, L_k, n_tiles;  // n_tiles = ceil(L_k / 128)
+  float* inv_norm;      // [H, n_tiles * 128] scratch: 1 / max(|k|, 1e-12), 0 past the end of the cache
+  float* a_out;         // [H, L_k] softmax argument of the redundancy
+  float2* a_partial;    // [H, n_tiles * 4] (max, sum of exp) of a per 32 keys
+  uint32_t* status;
+};
+// a_j = column mean of the cosine matrix with zeroed diagonal (Eq. 11), or with `max_similarity` the largest
+// similarity of token j to another token; bf16 keys only
+int score_red_tiled(fc_ctx* ctx, cudaStream_t st, RedTiledArgs args, int d, int64_t k_hs, int64_t k_rs, const void* K,
+                    bool max_similarity);
+
 // Frame-level query granularity on tensor cores (bf16, one query head per key head): first every query's (maximum,
 // sum) over slices of the candidates into `ml_part` ([H, kScoreFrameMaxSlices, L_q] at most, log2 domain), their
 // merge into `nlse` ([H, L_q], minus the log2-domain log-sum-exp), then mass[h, j] = sum_i exp(q_i . k_j * scale -

@@ -530,6 +530,61 @@ def test_score_frame_level_accumulated_over_steps(ctx):
                                atol=1e-4 * np.abs(want["score"]).max())
 
 
+# Redundancy from explicit similarity tiles (Eq. 11 as written) and the column-maximum variant
+
+@pytest.mark.parametrize("d,L_k,keys", [(128, 1331, "clustered"), (64, 700, "normal"), (128, 4096, "normal"), (128, 130, "normal")])
+def test_score_tiled_redundancy_every_element(ctx, d, L_k, keys):
+    from paper_2602_10825_b200 import binding
+    w = wl.Workload("t", "bf16", H=2, d=d, W=1, n_c=100, B=L_k, L_k=L_k, seed=23, sigma=0.5, keys=keys)
+    Q, K, _ = wl.candidates(w)
+    K[1, 5] = 0  # a zero key: similarity 0 to everything
+    K[0, 9] = K[0, 2]  # an exact duplicate: similarity 1, and the diagonal must still be left out
+    for mode_g, mode_o in ((binding.RED_TILED, oracle.RED_PLAIN), (binding.RED_TILED_MAX, oracle.RED_MAXSIM)):
+        want = oracle.kv_score(wl.bits(Q), wl.bits(K), lambda_=0.07, pool_k=7, red_mode=mode_o)
+        red = torch.empty((2, L_k), device="cuda")
+        imp = torch.empty((2, L_k), device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        got = ctx.kv_score(dev(Q), dev(K), lambda_=0.07, pool_k=7, red=red, imp=imp, red_mode=mode_g, status=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        for name, g_, w_ in (("imp", imp, want["imp"]), ("red", red, want["red"]),
+                             ("score", got["score"], want["score"].astype(np.float64))):
+            g_ = g_.double().cpu().numpy()
+            assert (np.abs(g_ - w_) <= 1e-4 * np.abs(w_).max(axis=1, keepdims=True)).all(), (name, mode_g)
+    # the plain definition and the mean-key identity are the same function: both device modes agree as well
+    a = ctx.kv_score(dev(Q), dev(K), red_mode=binding.RED_TILED)["score"]
+    b = ctx.kv_score(dev(Q), dev(K), red_mode=binding.RED_MEANKEY)["score"]
+    assert (a - b).abs().max().item() <= 1e-4 * b.abs().max().item()
+
+
+def test_score_tiled_redundancy_full_size(ctx):
+    # config 3's compression event (24 heads x 23400 clustered keys) through the dense tiles: Red on every element
+    # against the oracle (which uses the mean-key identity at this size), and the softmax arguments of sampled
+    # columns against the plain definition evaluated column by column, for the mean and for the maximum
+    from paper_2602_10825_b200 import binding
+    w = wl.CONFIGS["cached_step_bf16"]
+    Q, K, _ = wl.candidates(w)
+    Kg, Qg = dev(K), dev(Q)
+    want = oracle.kv_score(wl.bits(Q), wl.bits(K), lambda_=w.lam, pool_k=w.pool_k)
+    cols = np.unique(np.concatenate([[0, 1, 127, 128, w.L_k - 1], np.random.default_rng(3).integers(0, w.L_k, 40)])).astype(np.int32)
+    for mode_g, mode_o in ((binding.RED_TILED, oracle.RED_PLAIN), (binding.RED_TILED_MAX, oracle.RED_MAXSIM)):
+        red = torch.empty((w.H, w.L_k), device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        got = ctx.kv_score(Qg, Kg, lambda_=w.lam, pool_k=w.pool_k, red=red, red_mode=mode_g, status=status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        r = red.double().cpu().numpy()
+        assert abs(r.sum(axis=1) - 1).max() < 1e-4
+        if mode_g == binding.RED_TILED:
+            assert (np.abs(r - want["red"]) <= 1e-4 * want["red"].max(axis=1, keepdims=True)).all()
+            assert np.abs(got["score"].double().cpu().numpy() - want["score"]).max() <= 1e-4 * np.abs(want["score"]).max()
+        # Red = softmax(a): differences of log Red between columns are differences of a
+        a = oracle.key_similarity_columns(wl.bits(K), cols, mode_o)
+        d_gpu = np.log(r[:, cols]) - np.log(r[:, cols[:1]])
+        d_orc = a - a[:, :1]
+        assert np.abs(d_gpu - d_orc).max() <= 1e-4, mode_g
+
+
 def test_score_gqa_and_d64(ctx):
     Q = wl.normal((4, 20, 64), 31, 1.0)
     K = wl.normal((2, 300, 64), 32, 1.0)

@@ -237,6 +237,7 @@ score_finalize_kernel(ScoreGeom g, const float* __restrict__ imp_in, const float
   __shared__ float sm_m[kFinThreads / 32], sm_l[kFinThreads / 32];
   __shared__ float sh_m, sh_l;
   const int hk = blockIdx.y, tid = threadIdx.x;
+  fc::pdl_wait();  // launched under the tail of the kernel that writes imp, a and the softmax statistics
   float m = -INFINITY, l = 0.f;
   for (int t = tid; t < g.n_partials; t += kFinThreads) {
     const float2 p = a_partial[hk * g.n_partials + t];
@@ -439,7 +440,7 @@ extern "C" int fc_kv_score(fc_ctx* ctx, void* stream, const fc_score_desc* desc,
     g.n_partials = g.n_tiles * 4;
   }
   // 3. softmax of the redundancy argument, max-pool of the importance, lambda-mix
-  score_finalize_kernel<<<dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), kFinThreads, 0, st>>>(g, imp_buf, w.a, w.a_partial, red, score);
-  FC_LAUNCH_CHECK("score_finalize_kernel");
+  FC_CUDA_CHECK(fc::launch_pdl(score_finalize_kernel, dim3((g.L_k + kFinKeys - 1) / kFinKeys, g.H_kv), dim3(kFinThreads), 0,
+                               st, g, (const float*)imp_buf, (const float*)w.a, (const float2*)w.a_partial, red, score));
   return FC_OK;
 }

@@ -107,6 +107,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
   }
+  // Both passes let their successor (pass 2, the finalize kernel) be scheduled under their tail; pass 2 is such a
+  // successor itself and waits here, its barriers already initialised, for pass 1's results to be complete.
+  fc::pdl_launch_dependents();
+  if (PASS == 2) fc::pdl_wait();
   if (PASS == 2 && tid < kNQ) {
     // log-sum-exp of query `tid` over the whole head: pass 1's per-slice (max, sum) pairs, merged in slice order
     float lse = INFINITY;  // padding queries: exp2(anything - inf) = 0
@@ -400,15 +404,20 @@ int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs g, int d, int64_t q_h
   g.n_slices = (g.n_tiles + g.tiles_per_slice - 1) / g.tiles_per_slice;  // no empty slice
   const size_t smem = (size_t)(1 + kRing) * kKeys * d * 2 + sizeof(TcSmem) + 1024;
   const dim3 grid(g.n_slices, g.H);
-  auto launch = [&](auto kernel, int threads) -> int {
+  auto launch = [&](auto kernel, int threads, bool dependent) -> int {
     FC_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    kernel<<<grid, threads, smem, st>>>(tq, tk, g);
-    FC_LAUNCH_CHECK("score_tc_kernel");
+    if (dependent) {
+      FC_CUDA_CHECK(launch_pdl(kernel, grid, dim3(threads), smem, st, tq, tk, g));
+    } else {
+      kernel<<<grid, threads, smem, st>>>(tq, tk, g);
+      FC_LAUNCH_CHECK("score_tc_kernel");
+    }
     return FC_OK;
   };
-  if ((rc = d == 128 ? launch(score_tc_kernel<128, 1>, kThreadsOf<1>) : launch(score_tc_kernel<64, 1>, kThreadsOf<1>)) != FC_OK)
+  if ((rc = d == 128 ? launch(score_tc_kernel<128, 1>, kThreadsOf<1>, false)
+                     : launch(score_tc_kernel<64, 1>, kThreadsOf<1>, false)) != FC_OK)
     return rc;
-  return d == 128 ? launch(score_tc_kernel<128, 2>, kThreadsOf<2>) : launch(score_tc_kernel<64, 2>, kThreadsOf<2>);
+  return d == 128 ? launch(score_tc_kernel<128, 2>, kThreadsOf<2>, true) : launch(score_tc_kernel<64, 2>, kThreadsOf<2>, true);
 }
 
 }  // namespace fc

@@ -1,16 +1,18 @@
 // fc_kv_select_compact: per-head top-B of the selection score (text after Eq. 12) and the
 // retention of the selected K/V rows (Sec. 3.3).
 //
-// Selection: one cluster of four 1024-thread blocks per head, each holding a quarter of the head's keys.  Scores become order-preserving 32-bit keys (NaN
-// ranks as -inf, -0 as +0) held in shared memory when they fit; an 8-bit-digit radix select over
-// the bits in which the head's keys differ (at most 4 passes) finds the key T of the B-th largest
-// score and how many keys exceed it; one ordered
+// Selection: one cluster of up to four 1024-thread blocks per head, each holding its share of the head's keys.
+// Scores become order-preserving 32-bit keys (NaN ranks as -inf, -0 as +0) held in shared memory when they fit; an
+// 11-bit-digit radix select over the bits in which the head's keys differ (at most 3 passes, one cluster barrier
+// each) finds the key T of the B-th largest score and how many keys exceed it; one ordered
 // compaction then keeps every key above T plus the lowest-index keys equal to T, so the kept
 // set is exactly the first B elements of the total order (score descending, index ascending),
 // written in ascending index order.  Integer work only: bit-exact.
 //
 // Compaction: a separate streaming kernel moves whole rows with 16-byte accesses, several
-// independent loads in flight per thread; rows that were dropped are never read.
+// independent loads in flight per thread; rows that were dropped are never read.  It is launched as a programmatic
+// dependent of the selection: its blocks take their places on the SMs while the selection still runs and start
+// copying the moment it has ended.
 #include <cooperative_groups.h>
 
 #include "fc_common.cuh"
@@ -27,16 +29,18 @@ __device__ __forceinline__ uint32_t score_key(float s, bool& is_nan) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);  // larger float <=> larger key
 }
 
-// One cluster of kSelCluster CTAs per head; CTA r of the cluster owns the contiguous index range
-// [r * chunk, (r + 1) * chunk) of the head.  The CTAs exchange their partial results (minimum / maximum, digit
-// histograms, counts of kept keys) by reading each other's shared memory.
-constexpr int kSelCluster = 4;
+// One cluster of CTAs per head (1, 2 or 4 of them: as many as keep the whole grid within one wave); CTA r of the
+// cluster owns the contiguous index range [r * chunk, (r + 1) * chunk) of the head.  The CTAs exchange their partial
+// results (minimum / maximum, digit histograms, counts of kept keys) by reading each other's shared memory.
+constexpr int kDigitBits = 11, kBins = 1 << kDigitBits;  // at most three passes over 32 bits
+constexpr int kMaxCluster = 4;  // measured: a cluster of 8 is slower (25 us against 19 on 12 heads x 20400 keys)
 
 struct SelShared {
-  uint32_t hist[4][256];   // four copies, one per quarter of the warps, to spread the atomics
-  uint32_t hist_cta[256];  // this CTA's histogram of the current digit (read by the other CTAs)
+  uint32_t hist[2][kBins];      // two copies (even / odd warps) to spread the atomics
+  uint32_t hist_cta[2][kBins];  // this CTA's histogram of the current digit, read by the other CTAs; passes alternate
+                                // between the two buffers, so one cluster barrier per pass is enough
   uint32_t red_min[kSelThreads / 32], red_max[kSelThreads / 32];
-  uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32];
+  uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32], scan_w[kSelThreads / 32];
   uint32_t cta_min, cta_max, cta_gt, cta_eq;  // read by the other CTAs
   uint32_t prefix, remaining, nan;
 };
@@ -49,12 +53,15 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ uint32_t smem_keys[];
   __shared__ SelShared sh;
-  const int rank = (int)cluster.block_rank(), h = blockIdx.x / kSelCluster, tid = threadIdx.x;
+  const int cs = (int)cluster.num_blocks();
+  const int rank = (int)cluster.block_rank(), h = blockIdx.x / cs, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int begin = min(rank * chunk, L_k), n = min(begin + chunk, L_k) - begin;  // this CTA's keys: begin + [0, n)
   const float* s = score + (size_t)h * L_k + begin;
   int32_t* out = kept_idx + (size_t)h * B;  // B <= L_k here (the identity case is handled apart)
 
+  fc::pdl_launch_dependents();  // the gather's blocks may take their places; they wait for this grid to end
+  fc::pdl_wait();               // the scores are complete and visible from here on
   if (tid == 0) sh.nan = 0;
   if (tid == 0 && blockIdx.x == 0 && n_kept) *n_kept = B;
   __syncthreads();
@@ -94,18 +101,23 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
     sh.red_max[warp] = kmax;
   }
   __syncthreads();
-  if (tid == 0) {
-    for (int w = 0; w < kSelThreads / 32; ++w) {
-      kmin = min(kmin, sh.red_min[w]);
-      kmax = max(kmax, sh.red_max[w]);
+  if (warp == 0) {
+    kmin = sh.red_min[lane];
+    kmax = sh.red_max[lane];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+      kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
     }
-    sh.cta_min = kmin;
-    sh.cta_max = kmax;
+    if (lane == 0) {
+      sh.cta_min = kmin;
+      sh.cta_max = kmax;
+    }
   }
   cluster.sync();
   kmin = 0xffffffffu;
   kmax = 0;
-  for (int q = 0; q < kSelCluster; ++q) {
+  for (int q = 0; q < cs; ++q) {
     const SelShared* other = cluster.map_shared_rank(&sh, q);
     kmin = min(kmin, other->cta_min);
     kmax = max(kmax, other->cta_max);
@@ -118,60 +130,68 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
     return score_key(s[j], nn) - base;
   };
 
-  // Radix select, most significant digit first, 8 bits at a time over the n_bits that vary.  Invariant: the
+  // Radix select, most significant digit first, kDigitBits at a time over the n_bits that vary.  Invariant: the
   // B-th largest key has the bits of `prefix` above bit `hi`, and `remaining` of the keys with that prefix
   // (counted from the largest) are still to be taken.  Every CTA adds up all CTAs' histograms and takes the
   // same decision.
   uint32_t prefix = 0, remaining = (uint32_t)B;
-  for (int hi = n_bits; hi > 0;) {
-    const int lo = max(hi - 8, 0);
+  int pass = 0;
+  for (int hi = n_bits; hi > 0; ++pass) {
+    const int lo = max(hi - kDigitBits, 0);
     const uint32_t digit_mask = (1u << (hi - lo)) - 1u;
-    sh.hist[tid >> 8][tid & 255] = 0;
+    for (int b = tid; b < 2 * kBins; b += kSelThreads) (&sh.hist[0][0])[b] = 0;
     __syncthreads();
     for (int j = tid; j < n; j += kSelThreads) {
       const uint32_t k = key_at(j);
       const bool candidate = hi >= 32 || (k >> hi) == (prefix >> hi);
-      if (candidate) atomicAdd(&sh.hist[warp & 3][(k >> lo) & digit_mask], 1u);
+      if (candidate) atomicAdd(&sh.hist[warp & 1][(k >> lo) & digit_mask], 1u);
     }
     __syncthreads();
-    if (tid < 256) sh.hist_cta[tid] = (sh.hist[0][tid] + sh.hist[1][tid]) + (sh.hist[2][tid] + sh.hist[3][tid]);
+    uint32_t* mine = sh.hist_cta[pass & 1];
+    for (int b = tid; b < kBins; b += kSelThreads) mine[b] = sh.hist[0][b] + sh.hist[1][b];
     cluster.sync();
-    if (tid < 32) {
-      // digits from 255 downwards, eight per lane; the digit of the B-th largest key is where the running
+    {
+      // digits from the largest downwards, two per thread; the digit of the B-th largest key is where the running
       // count first reaches `remaining`
-      uint32_t c[8], tot = 0;
+      const int d0 = kBins - 1 - 2 * tid, d1 = d0 - 1;
+      uint32_t r0[kMaxCluster], r1[kMaxCluster];  // all remote loads in flight before the first add
 #pragma unroll
-      for (int i = 0; i < 8; ++i) c[i] = 0;
-      for (int q = 0; q < kSelCluster; ++q) {
-        const SelShared* other = cluster.map_shared_rank(&sh, q);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) c[i] += other->hist_cta[255 - (tid * 8 + i)];
+      for (int q = 0; q < kMaxCluster; ++q) {
+        const SelShared* other = cluster.map_shared_rank(&sh, q < cs ? q : 0);
+        r0[q] = other->hist_cta[pass & 1][d0];
+        r1[q] = other->hist_cta[pass & 1][d1];
       }
+      uint32_t c0 = 0, c1 = 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) tot += c[i];
+      for (int q = 0; q < kMaxCluster; ++q) {
+        c0 += q < cs ? r0[q] : 0u;
+        c1 += q < cs ? r1[q] : 0u;
+      }
+      const uint32_t tot = c0 + c1;
       uint32_t inc = tot;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
         const uint32_t v = __shfl_up_sync(0xffffffffu, inc, o);
-        if (tid >= o) inc += v;
+        if (lane >= o) inc += v;
       }
-      const uint32_t exc = inc - tot;
-      if (exc < remaining && remaining <= inc) {
-        uint32_t rem = remaining - exc;
-        int digit = 255 - tid * 8;
+      if (lane == 31) sh.scan_w[warp] = inc;
+      __syncthreads();
+      uint32_t before = lane < warp ? sh.scan_w[lane] : 0u;  // totals of the warps in front of this one
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (c[i] >= rem) {
-            digit = 255 - (tid * 8 + i);
-            break;
-          }
-          rem -= c[i];
+      for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xffffffffu, before, o);
+      const uint32_t exc = before + inc - tot;
+      if (exc < remaining && remaining <= exc + tot) {
+        uint32_t rem = remaining - exc;
+        int digit = d0;
+        if (c0 < rem) {
+          rem -= c0;
+          digit = d1;
         }
         sh.prefix = prefix | ((uint32_t)digit << lo);
         sh.remaining = rem;
       }
+      __syncthreads();
     }
-    cluster.sync();  // every CTA has read the histograms before the next pass clears them
     prefix = sh.prefix;
     remaining = sh.remaining;
     hi = lo;
@@ -202,10 +222,11 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
     sh.warp_eq[warp] = incl >> 16;
   }
   __syncthreads();
-  uint32_t base_gt = 0, base_eq = 0;
-  for (int w = 0; w < warp; ++w) {
-    base_gt += sh.warp_gt[w];
-    base_eq += sh.warp_eq[w];
+  uint32_t base_gt = lane < warp ? sh.warp_gt[lane] : 0u, base_eq = lane < warp ? sh.warp_eq[lane] : 0u;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {  // totals of the warps in front of this one
+    base_gt += __shfl_xor_sync(0xffffffffu, base_gt, o);
+    base_eq += __shfl_xor_sync(0xffffffffu, base_eq, o);
   }
   if (tid == kSelThreads - 1) {  // this CTA's totals, for the CTAs that own higher indices
     sh.cta_gt = base_gt + (incl & 0xffffu);
@@ -261,6 +282,7 @@ gather_rows_kernel(const uint8_t* __restrict__ K_src, const uint8_t* __restrict_
                    int64_t src_hs_b, int64_t src_rs_b, int64_t dst_hs_b, int64_t dst_rs_b,
                    uint32_t* __restrict__ status) {
   const int h = blockIdx.y;
+  fc::pdl_wait();  // the kept indices are complete and visible from here on
   const int64_t n_pieces = (int64_t)n_keep * pieces_per_row;
   const int64_t p0 = (int64_t)blockIdx.x * (kCopyThreads * kUnroll) + threadIdx.x;
   const int32_t* idx = kept_idx + (size_t)h * n_keep;
@@ -331,21 +353,26 @@ extern "C" int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* scor
     select_identity_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kept_idx, n_heads, L_k, score, n_kept, status);
     FC_LAUNCH_CHECK("select_identity_kernel");
   } else {
-    const int chunk = (L_k + kSelCluster - 1) / kSelCluster;
+    // cluster size: as many CTAs per head as keep all heads within one wave of the SMs
+    int cs = 1;
+    while (cs < kMaxCluster && n_heads * cs * 2 <= ctx->sm_count) cs *= 2;
+    const int chunk = (L_k + cs - 1) / cs;
     const size_t key_bytes = (size_t)chunk * 4;
     const bool smem_keys = key_bytes + sizeof(SelShared) + 1024 <= (size_t)ctx->smem_optin;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)n_heads * kSelCluster);
+    cfg.gridDim = dim3((unsigned)n_heads * cs);
     cfg.blockDim = dim3(kSelThreads);
     cfg.dynamicSmemBytes = smem_keys ? key_bytes : 0;
     cfg.stream = st;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = kSelCluster;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may be scheduled under the previous kernel's tail
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     if (smem_keys) {
       FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
@@ -360,10 +387,10 @@ extern "C" int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* scor
     const int ppr = d * es / 16;
     const int64_t n_pieces = (int64_t)n_keep * ppr;
     dim3 grid((unsigned)((n_pieces + kCopyThreads * kUnroll - 1) / (kCopyThreads * kUnroll)), n_heads);
-    gather_rows_kernel<<<grid, kCopyThreads, 0, st>>>(
-        (const uint8_t*)K_src, (const uint8_t*)V_src, (uint8_t*)K_dst, (uint8_t*)V_dst, kept_idx, n_keep,
-        L_k, ppr, strides->src_hs * es, strides->src_rs * es, strides->dst_hs * es, strides->dst_rs * es,
-        status);
+    FC_CUDA_CHECK(fc::launch_pdl(gather_rows_kernel, grid, dim3(kCopyThreads), 0, st, (const uint8_t*)K_src,
+                                 (const uint8_t*)V_src, (uint8_t*)K_dst, (uint8_t*)V_dst, (const int32_t*)kept_idx, n_keep,
+                                 L_k, ppr, strides->src_hs * es, strides->src_rs * es, strides->dst_hs * es,
+                                 strides->dst_rs * es, status));
     FC_LAUNCH_CHECK("gather_rows_kernel");
   }
   return FC_OK;

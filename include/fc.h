@@ -84,6 +84,14 @@ const char* fc_last_cuda_error(void);
 /* Number of SMs the context's persistent kernels size their grids by. */
 int fc_sm_count(const fc_ctx* ctx);
 
+/* Self-test of the bounded waits (no counterpart in the paper).  Every wait on a barrier inside the tensor-core
+ * kernels gives up after a wall-time limit instead of spinning forever; the kernel then runs to its normal end
+ * and sets FC_DEV_TIMEOUT.  This call launches one warp that waits, with the same routine and a limit of
+ * `limit_ns` (clamped to 1 us .. 1 s), on a barrier nobody signals.  After the caller's synchronisation `status`
+ * (DEVICE, required) has FC_DEV_TIMEOUT set and `waited_ns` (DEVICE [1] or NULL) holds how long the warp waited.
+ * Nothing faults or hangs; the context stays usable. */
+int fc_selftest_bounded_wait(fc_ctx* ctx, void* stream, uint64_t limit_ns, uint32_t* status, uint32_t* waited_ns);
+
 /* ------------------------------------------------------------------------------------------
  * fc_chunk_decide — per-chunk reuse decision.
  *

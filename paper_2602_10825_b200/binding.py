@@ -10,7 +10,8 @@ import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
-_LIB_PATH = os.path.join(_PKG, "libfc.so")
+# FC_LIB=debug selects the bounds-checking build (libfc_debug.so, see build.py); anything else the normal library
+_LIB_PATH = os.path.join(_PKG, "libfc_debug.so" if os.environ.get("FC_LIB") == "debug" else "libfc.so")
 _HEADER = os.path.join(_ROOT, "include", "fc.h")
 
 BF16, F32 = 0, 1
@@ -153,6 +154,12 @@ class Context:
             buf = torch.empty(n_bytes, dtype=torch.uint8, device=f"cuda:{self.device}")
             self._ws[key] = buf
         return buf
+
+    # ------------------------------------------------------------------ fc_selftest_bounded_wait
+    def selftest_bounded_wait(self, limit_ns, status, waited_ns=None):
+        rc = self._L.fc_selftest_bounded_wait(self._h, self._stream(), C.c_uint64(int(limit_ns)),
+                                              _dev(status, "status", torch.int32), _dev(waited_ns, "waited_ns", torch.int32))
+        self._check(rc, "fc_selftest_bounded_wait")
 
     # ------------------------------------------------------------------ fc_chunk_decide
     def chunk_decide(self, cur, prev, chunk_elem_off, chunk_step, warmup_m, eps, acc, *, force=None,

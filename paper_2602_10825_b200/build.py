@@ -10,6 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libfc.so")
+LIB_DEBUG = os.path.join(PKG, "libfc_debug.so")  # the same sources with -DFC_DEBUG_BOUNDS
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
@@ -19,19 +20,23 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB):
+def is_stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(ROOT, "include", "*.h"))
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ into one shared library.  Cross-compiles without a GPU."""
-    if not force and not is_stale():
-        return LIB
-    build_dir = os.path.join(PKG, "_build")
+def build(force: bool = False, verbose: bool = False, debug_bounds=None) -> str:
+    """Compile every .cu under csrc/ into one shared library.  Cross-compiles without a GPU.
+    debug_bounds=True builds libfc_debug.so, whose kernels guard their computed stores (see fc_common.cuh)."""
+    if debug_bounds is None:  # follow the variant the binding will load
+        debug_bounds = os.environ.get("FC_LIB") == "debug"
+    lib = LIB_DEBUG if debug_bounds else LIB
+    if not force and not is_stale(lib):
+        return lib
+    build_dir = os.path.join(PKG, "_build", "debug" if debug_bounds else "release")
     os.makedirs(build_dir, exist_ok=True)
     objs, procs = [], []
     for src in sources():
@@ -39,6 +44,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         objs.append(obj)
         cmd = [NVCC, *ARCH, "-lineinfo", "-O3", "-std=c++17",
                "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", src, "-o", obj]
+        if debug_bounds:
+            cmd.insert(1, "-DFC_DEBUG_BOUNDS")
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -50,9 +57,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed |= p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed")
-    subprocess.check_call([NVCC, *ARCH, "-shared", "-o", LIB] + objs + ["-lcudart_static", "-ldl", "-lrt", "-lpthread"])
-    return LIB
+    subprocess.check_call([NVCC, *ARCH, "-shared", "-o", lib] + objs + ["-lcudart_static", "-ldl", "-lrt", "-lpthread"])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug_bounds="--debug-bounds" in sys.argv))

@@ -561,7 +561,8 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
       ++items;
       tc_fence_after();
       const int row = it.row0 + x * kBM + r_in;
-      const bool row_ok = row < g.q_row_off[it.c + 1];
+      const bool row_ok = row < g.q_row_off[it.c + 1] &&
+                          fc::bounds_ok(row >= 0 && row < g.q_row_off[g.W] && it.h >= 0 && it.h < g.H_q, g.status);
       const float inv = l > 0.f ? 1.f / l : 0.f;
       __nv_bfloat16* out = O + (int64_t)it.h * g.o_hs + (int64_t)row * g.o_rs;
 #pragma unroll

@@ -40,6 +40,18 @@ inline int elem_size(int dtype) { return dtype == FC_F32 ? 4 : 2; }
     }                                               \
   } while (0)
 
+// Bounds-checking build (-DFC_DEBUG_BOUNDS, libfc_debug.so): every store whose address is computed from data read on
+// the device, or from a tile / slice walk, is guarded; a violated guard sets FC_DEV_BAD_INDEX in the status word and
+// skips the store (nothing traps).  In the normal build the guard is the constant `true`.
+#ifdef FC_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_ok(bool inside, uint32_t* status) {
+  if (!inside && status) atomicOr(status, (uint32_t)FC_DEV_BAD_INDEX);
+  return inside;
+}
+#else
+__device__ __forceinline__ bool bounds_ok(bool, uint32_t*) { return true; }
+#endif
+
 // Programmatic dependent launch.  launch_pdl() starts `kernel` so that its blocks may become resident while the
 // previous kernel of the stream is still running (once every block of that kernel has executed
 // pdl_launch_dependents() or exited); the kernel must execute pdl_wait() before it reads or writes anything the

@@ -267,7 +267,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       for (int i = wg; i < n; i += 2) {
         const int b = i & 1;
         const int tile_id = tile_of(i), j = tile_id * kKeys + row;  // this thread's key
-        const bool valid = j < g.L_k;
+        const bool valid = j < g.L_k && fc::bounds_ok(j >= 0 && hk >= 0 && hk < g.H && tile_id < g.n_tiles, g.status);
         const int64_t o = (int64_t)hk * g.L_k + j;
         const float n2 = valid && g.accum_phase != 1 ? g.norm2[o] : 0.f;  // in flight while the logits arrive
         mbar_wait_bounded(smem_u32(&sh->s_full[b]), (i >> 1) & 1, abort);

@@ -243,10 +243,11 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
   for (int j = j0; j < j1; ++j) {
     const uint32_t k = key_at(j);
     if (k > T) {
-      out[gt_before + min(eq_before, need_eq)] = begin + j;
+      const uint32_t pos = gt_before + min(eq_before, need_eq);
+      if (fc::bounds_ok(pos < (uint32_t)B, status)) out[pos] = begin + j;
       ++gt_before;
     } else if (k == T) {
-      if (eq_before < need_eq) out[gt_before + eq_before] = begin + j;
+      if (eq_before < need_eq && fc::bounds_ok(gt_before + eq_before < (uint32_t)B, status)) out[gt_before + eq_before] = begin + j;
       ++eq_before;
     }
   }
@@ -303,6 +304,10 @@ gather_rows_kernel(const uint8_t* __restrict__ K_src, const uint8_t* __restrict_
       }
       const int64_t so = (int64_t)h * src_hs_b + (int64_t)src_row * src_rs_b + c * 16;
       dst_off[u] = (int64_t)h * dst_hs_b + (int64_t)r * dst_rs_b + c * 16;
+      if (!fc::bounds_ok(r < n_keep && c < pieces_per_row, status)) {
+        ok[u] = false;
+        continue;
+      }
       kv[u] = fc::ld_stream16(K_src + so);
       vv[u] = fc::ld_stream16(V_src + so);
     }

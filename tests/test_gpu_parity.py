@@ -716,6 +716,79 @@ def test_pipeline_gpu_scores_feed_gpu_select(ctx):
     assert overlap > 0.99
 
 
+# ------------------------------------------------------------------------------------ canaries
+
+class _Guarded:
+    """Device buffers with canary elements in front of and behind the part a call may write."""
+
+    def __init__(self):
+        self.bufs = []
+
+    def flat(self, n, dtype, pad=64, fill=0):
+        buf = torch.full((n + 2 * pad,), 113, dtype=dtype, device="cuda")
+        buf[pad:pad + n] = fill
+        self.bufs.append((buf, pad, n))
+        return buf[pad:pad + n]
+
+    def rows(self, H, R, d, dtype):
+        """[H, R, d] view with one canary row before and after every head's rows."""
+        buf = torch.full((H, R + 2, d), 113, dtype=dtype, device="cuda")
+        self.bufs.append((buf, None, R))
+        return buf[:, 1:R + 1]
+
+    def check(self):
+        for buf, pad, n in self.bufs:
+            if pad is None:
+                assert (buf[:, 0] == 113).all() and (buf[:, n + 1] == 113).all()
+            else:
+                assert (buf[:pad] == 113).all() and (buf[pad + n:] == 113).all()
+
+
+def test_outputs_stay_inside_their_buffers(ctx):
+    # every output of every call sits between canaries, on ragged sizes (nothing a multiple of a tile)
+    g = _Guarded()
+    w = wl.Workload("c", "bf16", H=3, d=128, W=3, n_c=333, B=211, L_k=544, seed=77, sigma=0.5, keys="clustered")
+    n_el = w.n_c * w.hidden
+    off = np.arange(w.W + 1, dtype=np.int64) * n_el
+    cur, prev = wl.indicator_pair(w.W, n_el, [0.3, 0.01, 0.3], 5)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dec = ctx.chunk_decide(dev(cur), dev(prev), off, i32([4] * w.W), 1, 0.1, g.flat(w.W, torch.float32),
+                           l1rel=g.flat(w.W, torch.float32), recompute=g.flat(w.W, torch.uint8),
+                           active_ids=g.flat(w.W, torch.int32), n_active=g.flat(1, torch.int32), status=status)
+    y, cache = g.flat(w.W * n_el, torch.bfloat16), g.flat(w.W * n_el, torch.bfloat16)
+    ctx.chunk_cache_apply(dev(cur), y, cache, off, dec["recompute"], status=status)
+    Q, K, V = wl.qkv(w)
+    q_off, vis, slo, spo = wl.prefix_layout(w)
+    O = g.rows(w.H, w.window_rows, w.d, torch.bfloat16)
+    lse = g.rows(w.H, w.window_rows, 1, torch.float32)[:, :, 0]
+    ctx.chunk_attention(dev(Q), dev(K), dev(V), q_off, vis, slo, spo, dec["active_ids"], dec["n_active"], O, lse=lse,
+                        status=status)
+    Q_obs, Kc, Vc = wl.candidates(w)
+    outs = {k: g.flat(w.H * w.L_k, torch.float32).view(w.H, w.L_k) for k in ("imp", "red", "score")}
+    ctx.kv_score(dev(Q_obs), dev(Kc), status=status, **outs)
+    ctx.kv_score(dev(Q_obs), dev(Kc), status=status, red_mode=1, **outs)
+    kept = g.flat(w.H * w.B, torch.int32).view(w.H, w.B)
+    ctx.kv_select_compact(outs["score"], w.B, dev(Kc), dev(Vc), g.rows(w.H, w.B, w.d, torch.bfloat16),
+                          g.rows(w.H, w.B, w.d, torch.bfloat16), kept_idx=kept, n_kept=g.flat(1, torch.int32), status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    g.check()
+    assert dec["recompute"].cpu().tolist() == [1, 0, 1] and int(kept.max().item()) < w.L_k
+
+
+def test_a_wait_that_nobody_ends_gives_up_and_reports_it(ctx):
+    # the bounded wait of the tensor-core kernels, made to run out on purpose: one warp waits 1 ms for a barrier that
+    # is never signalled, returns, and the status word says so; the context keeps working afterwards
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.selftest_bounded_wait(1_000_000, status, waited)
+    torch.cuda.synchronize()
+    assert status.item() == 1  # FC_DEV_TIMEOUT
+    assert 0.9e6 <= waited.item() <= 50e6
+    w = wl.CONFIGS["tiny_f32"]
+    _attention_case(ctx, w, [0, 2], atol=1e-4, rel_l2=1e-4)
+
+
 # ------------------------------------------------------------------------------------ error conventions
 
 def test_bad_arguments_return_a_status_and_launch_nothing(ctx):

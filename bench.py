@@ -549,6 +549,27 @@ def time_cache_apply(step, iters=10):
     return ms, 3 * step.cur.numel() * step.cur.element_size()
 
 
+def time_token_map_attention(step, iters=5):
+    """fc_chunk_attention of all chunks with the K/V store read through a per-head token map (tile::gather4 loads)
+    instead of the segment table: the clean region is a sorted random subset of the candidate rows, as a top-B
+    selection leaves it, the window follows.  Returns ms per call."""
+    w, dev = step.w, step.device
+    g = torch.Generator(device=dev)
+    g.manual_seed(99)
+    n_clean = step.n_keep if w.B > 0 else 0
+    parts = []
+    if n_clean:
+        pick = torch.rand(w.H, step.L_k, generator=g, device=dev).argsort(dim=1)[:, :n_clean].sort(dim=1).values
+        parts.append(pick.to(torch.int32))
+    parts.append((w.B + torch.arange(w.window_rows, device=dev, dtype=torch.int32)).repeat(w.H, 1))
+    tok = torch.cat(parts, dim=1).contiguous()
+    act = torch.arange(w.W, dtype=torch.int32, device=dev)
+    n_act = torch.full((1,), w.W, dtype=torch.int32, device=dev)
+    fn = lambda: step.ctx.chunk_attention(step.Q, step.K, step.V, step.q_off, step.vis, None, None, act, n_act, step.O,
+                                          kv_token_index=tok, impl=2, status=step.status)
+    return time_calls(fn, iters, 2)
+
+
 def time_single_step_attention(ctx, device, iters=20):
     """The attention kernel alone on the single-step configuration (16 heads, 4 x 6240 tokens, no clean region):
     short enough to run at burst clocks.  Returns (ms, algorithmic FLOPs)."""
@@ -697,6 +718,13 @@ def main():
                 "frac": ca_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic("cache_apply_kernel", w.name), "ms": ca_ms,
                 "kernel": "cache_apply_kernel (fc_chunk_cache_apply, outside the timed step, every other chunk served "
                           "from the cache); algorithmic bytes = 3 x elements x element size", "peak_kind": peak_kind}
+            tm_ms = time_token_map_attention(step)
+            tm_tf = w.attention_flops(range(w.W)) / (tm_ms * 1e-3) / 1e12
+            line["attention_token_map"] = {
+                "bound": "tensor", "achieved": tm_tf, "peak": tensor_peak, "unit": "TFLOP/s", "frac": tm_tf / tensor_peak,
+                "ms": tm_ms, "segment_table_ms": stage_ms["attention"],
+                "kernel": "attention_ws_kernel<D, gather> (all chunks active, K/V rows fetched by tile::gather4 through a "
+                          "per-head token map; outside the timed step)", "peak_kind": peak_kind}
             if single is not None:
                 a_ms, a_flops = single
                 a_tf = a_flops / (a_ms * 1e-3) / 1e12

@@ -8,7 +8,9 @@
 //   warps 4-7  softmax of tile B
 //   warp  8    scheduler + TMA       takes the next item off the counter, publishes it to the
 //                                    other warps through a 2-slot ring, then loads the Q pair and
-//                                    streams K and V tiles into 2-stage rings
+//                                    streams K and V tiles into 2-stage rings (segment table: one tiled
+//                                    load per 64-column block; per-head token map: every lane gathers four
+//                                    rows at a time by index, tile::gather4, into the same swizzled tile)
 //   warps 9,10 MMA issuers           one thread per query tile
 //   warp  11   tail patcher          zeroes the rows of a V stage that lie past the end of a segment
 // Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
@@ -134,7 +136,9 @@ __device__ __forceinline__ void warp_wait(uint32_t bar, uint32_t parity, volatil
   mbar_wait_bounded(bar, parity, abort);
 }
 
-template <int D>
+// kGather: the logical key/value tokens are reached through the per-head token map g.tok_index (tmap_k / tmap_v are
+// then 2-D maps over all rows of all heads, box one row high) instead of the segment table.
+template <int D, bool kGather>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ fc::AttnGeom g,
@@ -277,6 +281,41 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             tma_load_3d(q_s + t * kTileBytes + x * kAtomBytes, &tmap_q, smem_u32(&sh->q_full), x * 64,
                         it.row0 + t * kBM, it.h);
       }
+      if constexpr (kGather) {
+        // One logical segment [0, n_vis) whose token j of head hk lives in physical row tok[j].  Lane L brings rows
+        // 4L .. 4L+3 of every tile; positions past the visible prefix repeat its last token (their logits are masked
+        // and their V rows zeroed like any other tail).  A row index outside the store is reported and replaced by 0.
+        const int32_t* tok = g.tok_index + (int64_t)it.hk * g.tok_hs;
+        const int k_base = (int)(it.hk * (g.k_hs / g.k_rs)), v_base = (int)(it.hk * (g.v_hs / g.v_rs));
+        for (int j0 = 0; j0 < it.n_vis; j0 += kBN, ++kv) {
+          const int st = kv % kStages, ph = (kv / kStages) & 1;
+          int r[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            r[e] = __ldg(tok + min(j0 + 4 * lane + e, it.n_vis - 1));  // in flight during the wait for the stage
+          }
+          warp_wait(smem_u32(&sh->k_empty[st]), ph ^ 1, abort);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (r[e] < 0 || r[e] >= g.kv_rows) {
+              if (g.status) atomicOr(g.status, FC_DEV_BAD_INDEX);
+              r[e] = 0;
+            }
+          }
+          if (lane == 0) mbar_expect_tx(smem_u32(&sh->k_full[st]), kTileBytes);
+          __syncwarp();
+          for (int x = 0; x < kAtoms; ++x)
+            tma_gather4_2d(k_s + st * kTileBytes + x * kAtomBytes + lane * 512, &tmap_k, smem_u32(&sh->k_full[st]), x * 64,
+                           k_base + r[0], k_base + r[1], k_base + r[2], k_base + r[3]);
+          warp_wait(smem_u32(&sh->v_empty[st]), ph ^ 1, abort);
+          if (lane == 0) mbar_expect_tx(smem_u32(&sh->v_full[st]), kTileBytes);
+          __syncwarp();
+          for (int x = 0; x < kAtoms; ++x)
+            tma_gather4_2d(v_s + st * kTileBytes + x * kAtomBytes + lane * 512, &tmap_v, smem_u32(&sh->v_full[st]), x * 64,
+                           v_base + r[0], v_base + r[1], v_base + r[2], v_base + r[3]);
+          __syncwarp();
+        }
+      } else {
       for (int s = 0; s < g.n_seg; ++s) {
         const int seg_vis = min(g.seg_log[s + 1], it.n_vis) - g.seg_log[s];
         if (seg_vis <= 0) break;
@@ -298,6 +337,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           }
           __syncwarp();
         }
+      }
       }
       ++it_n;
     }
@@ -618,13 +658,15 @@ int attention_ws_launch(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const C
   // at least half of the shared memory, so that a second CTA (and its 512 columns) never joins the SM
   const size_t need = (2 + 2 * kStages) * (size_t)kBM * g.d * 2 + sizeof(WsSmem) + 1024;
   const size_t smem = std::max<size_t>(need, 120 * 1024);
-  if (g.d == 128) {
-    FC_CUDA_CHECK(cudaFuncSetAttribute(attention_ws_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attention_ws_kernel<128><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O, counter);
-  } else {
-    FC_CUDA_CHECK(cudaFuncSetAttribute(attention_ws_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    attention_ws_kernel<64><<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O, counter);
-  }
+  auto launch = [&](auto kernel) -> int {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<grid, kThreads, smem, st>>>(tq, tk, tv, g, (__nv_bfloat16*)O, counter);
+    return FC_OK;
+  };
+  int rc;
+  if (g.tok_index) rc = g.d == 128 ? launch(attention_ws_kernel<128, true>) : launch(attention_ws_kernel<64, true>);
+  else rc = g.d == 128 ? launch(attention_ws_kernel<128, false>) : launch(attention_ws_kernel<64, false>);
+  if (rc != FC_OK) return rc;
   FC_LAUNCH_CHECK("attention_ws_kernel");
   return FC_OK;
 }

@@ -277,6 +277,89 @@ def test_attention_token_index_map(ctx):
     _attention_case(ctx, w, [0, 1], token_map=True, atol=1e-4, rel_l2=1e-4)
     wb = wl.Workload("m", "bf16", H=2, d=128, W=2, n_c=96, B=50, L_k=146, seed=14, sigma=0.5)
     _attention_case(ctx, wb, [1], token_map=True, atol=1e-2, rel_l2=1e-2)
+    _attention_case(ctx, wb, [0, 1], token_map=True, impl=2, atol=1e-2, rel_l2=1e-2)  # on the tensor cores: gathered rows
+
+
+@pytest.mark.parametrize("d", [128, 64])
+def test_attention_token_index_map_tensor_cores(ctx, d):
+    # bf16 through a per-head token map on the tcgen05 kernel: several key tiles with a ragged end, visible lengths that
+    # are not multiples of four, grouped query heads (two query heads share a map), every physical row that no token
+    # maps to filled with NaN / infinities / 3e38, a chunk that sees nothing and a chunk that sees one token
+    H_q, H_kv, L_log, L_phys = 4, 2, 777, 1500
+    rng = np.random.default_rng(21)
+    tok = np.stack([rng.permutation(L_phys)[:L_log] for _ in range(H_kv)]).astype(np.int32)
+    Q = wl.normal((H_q, 600, d), 71, 0.5, torch.bfloat16)
+    K = wl.normal((H_kv, L_phys, d), 72, 0.5, torch.bfloat16)
+    V = wl.normal((H_kv, L_phys, d), 73, 0.5, torch.bfloat16)
+    bad = torch.tensor([float("nan"), float("inf"), -float("inf"), 3e38, -3e38]).to(torch.bfloat16)
+    for h in range(H_kv):
+        unused = np.setdiff1d(np.arange(L_phys), tok[h])
+        K[h, unused] = bad[torch.arange(len(unused)) % 5][:, None]
+        V[h, unused] = bad[(torch.arange(len(unused)) + 2) % 5][:, None]
+    q_off = np.array([0, 130, 131, 400, 600], np.int32)
+    vis = np.array([L_log, 1, 0, 389], np.int32)
+    O0 = wl.normal((H_q, 600, d), 74, 1.0, torch.bfloat16)
+    Og = dev(O0).clone()
+    lse_g = torch.full((H_q, 600), float("nan"), device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    active = [0, 1, 2, 3]
+    ctx.chunk_attention(dev(Q), dev(K), dev(V), q_off, vis, None, None, i32(active), i32([4]), Og, lse=lse_g,
+                        kv_token_index=i32(tok), impl=2, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    O_want, lse_want = oracle.chunk_attention(wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, None, None, active,
+                                              kv_token_index=tok, O_init=O0.double().numpy())
+    got = Og.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    assert np.abs(got - O_want).max() <= 1e-2
+    assert np.linalg.norm(got - O_want) <= 1e-2 * np.linalg.norm(O_want)
+    lg = lse_g.double().cpu().numpy()
+    fin = np.isfinite(lse_want)
+    np.testing.assert_allclose(lg[fin], lse_want[fin], atol=2e-3)
+    assert np.array_equal(np.isneginf(lg), np.isneginf(lse_want))
+    # an index outside the store is reported, not followed
+    tok_bad = tok.copy()
+    tok_bad[1, 5] = L_phys + 7
+    ctx.chunk_attention(dev(Q), dev(K), dev(V), q_off, vis, None, None, i32(active), i32([4]), Og, kv_token_index=i32(tok_bad),
+                        impl=2, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 4  # FC_DEV_BAD_INDEX
+
+
+def test_attention_through_the_kept_index_map_at_full_size(ctx):
+    # config 3: instead of compacting the 23400-token history to the 18720 kept tokens and attending over the compact
+    # copy, attend over the uncompacted store through the per-head kept-index list (the window chunks follow the
+    # history in the same store).  Sampled rows against the oracle, and against the compact-then-attend result.
+    w = wl.CONFIGS["cached_step_bf16"]
+    H, d, n_hist = w.H, w.d, w.L_k
+    rng = np.random.default_rng(8)
+    K = wl.clustered_keys(H, n_hist + w.window_rows, d, 9001)
+    V = wl.normal((H, n_hist + w.window_rows, d), 9002, w.sigma, torch.bfloat16)
+    Q = wl.normal((H, w.window_rows, d), 9003, w.sigma, torch.bfloat16)
+    kept = np.stack([np.sort(rng.choice(n_hist, w.B, replace=False)) for _ in range(H)]).astype(np.int32)
+    tok = np.concatenate([kept, np.tile(n_hist + np.arange(w.window_rows, dtype=np.int32), (H, 1))], axis=1)
+    q_off, vis, _, _ = wl.prefix_layout(w)
+    active = [2, 5, 7]
+    rows = wl.sample_rows(w, 192, 5, chunks=active)
+    Kg, Vg, Qg = dev(K), dev(V), dev(Q)
+    O_map = torch.zeros((H, w.window_rows, d), dtype=torch.bfloat16, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.chunk_attention(Qg, Kg, Vg, q_off, vis, None, None, i32(active + [-1] * 5), i32([3]), O_map,
+                        kv_token_index=i32(tok), impl=2, status=status)
+    # the same through a compact copy [kept history | window] and the segment table
+    idx = torch.as_tensor(tok, dtype=torch.long, device="cuda")[:, :, None].expand(H, tok.shape[1], d)
+    Kc, Vc = torch.gather(Kg, 1, idx), torch.gather(Vg, 1, idx)
+    _, _, slo, spo = wl.prefix_layout(w)
+    O_cmp = torch.zeros_like(O_map)
+    ctx.chunk_attention(Qg, Kc, Vc, q_off, vis, slo, spo, i32(active + [-1] * 5), i32([3]), O_cmp, impl=2, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert (O_map.float() - O_cmp.float()).abs().max().item() <= 2e-3  # same arithmetic, other addressing
+    O_want, _ = oracle.chunk_attention(wl.bits(Q), wl.bits(K), wl.bits(V), q_off, vis, None, None, active,
+                                       kv_token_index=tok, sample_rows=rows)
+    got = O_map[:, torch.as_tensor(rows, dtype=torch.long, device="cuda")].double().cpu().numpy()
+    assert np.abs(got - O_want).max() <= 1e-2
+    assert np.linalg.norm(got - O_want) <= 1e-2 * np.linalg.norm(O_want)
 
 
 @pytest.mark.parametrize("d", [128, 64])
@@ -363,7 +446,7 @@ def _poison_unreferenced_rows(K, V, vis_max, slo, spo):
 
 
 @pytest.mark.parametrize("d", [128, 64])
-def test_attention_ignores_rows_outside_the_visible_segments(ctx, d):
+def test_attention_ignores_rows_outside_the_visible_segments(ctx, d, impl=2):
     # The K/V buffer of the method has slots that are not written yet, and a segment's last 128-row tile drags in
     # whatever follows the segment.  Every such row is filled with NaN, infinities and 3e38 here: the outputs must
     # still match the oracle (which never reads those rows) and be finite.
@@ -384,7 +467,7 @@ def test_attention_ignores_rows_outside_the_visible_segments(ctx, d):
     q_off = np.array([0, 130, 400, 700], np.int32)
     vis = np.array([slo[-1], 700, 166], np.int32)
     assert _poison_unreferenced_rows(K, V, int(slo[-1]), slo, phys) > 100
-    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, phys.astype(np.int32), [0, 1, 2], 2)
+    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, phys.astype(np.int32), [0, 1, 2], impl)
     assert torch.isfinite(Og.float()).all()
     # (2) the prefix layout [clean region | gap | chunk 0 | gap | chunk 1 | unwritten rest], the second chunk's slot
     # only partly written: chunk 1 sees 100 of its 328 rows, the other 228 are poison inside its own segment
@@ -398,17 +481,17 @@ def test_attention_ignores_rows_outside_the_visible_segments(ctx, d):
     q_off = np.array([0, n_c, 2 * n_c], np.int32)
     vis = np.array([B + n_c, B + n_c + 100], np.int32)
     assert _poison_unreferenced_rows(K, V, int(vis[1]), slo, spo) > 400
-    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, spo, [0, 1], 2)
+    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, spo, [0, 1], impl)
     assert torch.isfinite(Og.float()).all()
     # the CUDA-core kernel reads through the same tables
     Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, spo, [0, 1], 1)
     assert torch.isfinite(Og.float()).all()
 
 
-def test_attention_bf16_many_items_per_cta(ctx):
+def test_attention_bf16_many_items_per_cta(ctx, impl=2):
     # more work items than SMs, of very different lengths: exercises the device-side item queue
     w = wl.Workload("q", "bf16", H=40, d=128, W=6, n_c=520, B=300, L_k=820, seed=18, sigma=0.5)
-    _attention_case(ctx, w, [0, 1, 3, 5], impl=2, sample=wl.sample_rows(w, 40, 1), atol=1e-2, rel_l2=1e-2)
+    _attention_case(ctx, w, [0, 1, 3, 5], impl=impl, sample=wl.sample_rows(w, 40, 1), atol=1e-2, rel_l2=1e-2)
 
 
 # The launch configurations the benchmark times, at full size, on sampled query rows over the full key range:

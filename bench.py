@@ -718,6 +718,21 @@ def main():
                 "frac": ca_gbs / peaks["hbm_gbs"], "traffic": ncu_traffic("cache_apply_kernel", w.name), "ms": ca_ms,
                 "kernel": "cache_apply_kernel (fc_chunk_cache_apply, outside the timed step, every other chunk served "
                           "from the cache); algorithmic bytes = 3 x elements x element size", "peak_kind": peak_kind}
+            score2 = torch.empty_like(step.score)
+            base_ms = time_calls(lambda: step.ctx.kv_score(step.Q_obs, step.K_cand, lambda_=w.lam, pool_k=w.pool_k,
+                                                           score=score2, status=step.status), 5, 2)
+            rt_ms = time_calls(lambda: step.ctx.kv_score(step.Q_obs, step.K_cand, lambda_=w.lam, pool_k=w.pool_k,
+                                                         score=score2, red_mode=1, status=step.status), 5, 2)
+            rt_flops = 2.0 * step.L_k * step.L_k * w.d * w.H
+            rt_tf = rt_flops / ((rt_ms - base_ms) * 1e-3) / 1e12
+            line["roofline_red_tiled"] = {
+                "bound": "tensor", "achieved": rt_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": rt_tf / peaks["bf16_tflops"], "traffic": ncu_traffic("red_tiled_kernel", w.name),
+                "ms": rt_ms - base_ms, "call_ms": rt_ms,
+                "kernel": "red_tiled_kernel + key_inv_norm_kernel (red_mode = tiled: the cosine-similarity matrix in "
+                          "128 x 128 tcgen05 tiles, never stored); time = fc_kv_score in tiled mode minus the same call "
+                          "in mean-key mode; FLOPs = 2 L_k^2 d H, the dense work the mean-key identity avoids: "
+                          "reported apart, not part of the score stage's figure", "peak_kind": peak_kind + " burst"}
             tm_ms = time_token_map_attention(step)
             tm_tf = w.attention_flops(range(w.W)) / (tm_ms * 1e-3) / 1e12
             line["attention_token_map"] = {

@@ -12,7 +12,8 @@
 //                                    load per 64-column block; per-head token map: every lane gathers four
 //                                    rows at a time by index, tile::gather4, into the same swizzled tile)
 //   warps 9,10 MMA issuers           one thread per query tile
-//   warp  11   tail patcher          zeroes the rows of a V stage that lie past the end of a segment
+//   warp  11   tail patcher          zeroes the rows of a V stage that lie past the end of a segment (with a token
+//                                    map it also gathers the V rows, so that two warps share the copy instructions)
 // Tensor memory: S_A [0,128) S_B [128,256) O_A [256,384) O_B [384,512).
 // A key tile of 128 tokens is worked through as two halves of 64: S_x is two 64-column accumulators, each with
 // its own "full" and "P ready" barriers, and P (bf16) of a half overwrites the first 32 columns of that half.
@@ -286,7 +287,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         // 4L .. 4L+3 of every tile; positions past the visible prefix repeat its last token (their logits are masked
         // and their V rows zeroed like any other tail).  A row index outside the store is reported and replaced by 0.
         const int32_t* tok = g.tok_index + (int64_t)it.hk * g.tok_hs;
-        const int k_base = (int)(it.hk * (g.k_hs / g.k_rs)), v_base = (int)(it.hk * (g.v_hs / g.v_rs));
+        const int k_base = (int)(it.hk * (g.k_hs / g.k_rs));
         for (int j0 = 0; j0 < it.n_vis; j0 += kBN, ++kv) {
           const int st = kv % kStages, ph = (kv / kStages) & 1;
           int r[4];
@@ -307,13 +308,7 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
           for (int x = 0; x < kAtoms; ++x)
             tma_gather4_2d(k_s + st * kTileBytes + x * kAtomBytes + lane * 512, &tmap_k, smem_u32(&sh->k_full[st]), x * 64,
                            k_base + r[0], k_base + r[1], k_base + r[2], k_base + r[3]);
-          warp_wait(smem_u32(&sh->v_empty[st]), ph ^ 1, abort);
-          if (lane == 0) mbar_expect_tx(smem_u32(&sh->v_full[st]), kTileBytes);
-          __syncwarp();
-          for (int x = 0; x < kAtoms; ++x)
-            tma_gather4_2d(v_s + st * kTileBytes + x * kAtomBytes + lane * 512, &tmap_v, smem_u32(&sh->v_full[st]), x * 64,
-                           v_base + r[0], v_base + r[1], v_base + r[2], v_base + r[3]);
-          __syncwarp();
+          __syncwarp();  // (the V rows of the tile are gathered by warp 11: two warps issue the copies)
         }
       } else {
       for (int s = 0; s < g.n_seg; ++s) {
@@ -486,6 +481,23 @@ attention_ws_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         for (int j0 = 0; j0 < seg_vis; j0 += kBN, ++kv) {
           const int st = kv % kStages, ph = (kv / kStages) & 1;
           const int cols_valid = min(kBN, seg_vis - j0);
+          if constexpr (kGather) {
+            // token map: this warp also brings the tile's V rows (lane L rows 4L .. 4L+3, as the copy warp does for K)
+            const int32_t* tok = g.tok_index + (int64_t)it.hk * g.tok_hs;
+            const int v_base = (int)(it.hk * (g.v_hs / g.v_rs));
+            int r[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) r[e] = __ldg(tok + min(j0 + 4 * lane + e, it.n_vis - 1));
+            warp_wait(smem_u32(&sh->v_empty[st]), ph ^ 1, abort);
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              if (r[e] < 0 || r[e] >= g.kv_rows) r[e] = 0;  // reported by the copy warp, which reads the same indices
+            if (lane == 0) mbar_expect_tx(smem_u32(&sh->v_full[st]), kTileBytes);
+            __syncwarp();
+            for (int x = 0; x < kAtoms; ++x)
+              tma_gather4_2d(v_s + st * kTileBytes + x * kAtomBytes + lane * 512, &tmap_v, smem_u32(&sh->v_full[st]),
+                             x * 64, v_base + r[0], v_base + r[1], v_base + r[2], v_base + r[3]);
+          }
           warp_wait(smem_u32(&sh->v_full[st]), ph, abort);
           if (cols_valid < kBN) {
             uint8_t* vt = v_tiles + st * kTileBytes;

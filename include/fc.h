@@ -145,9 +145,10 @@ int fc_chunk_decide(fc_ctx* ctx, void* stream, const void* cur, const void* prev
  *   - Limit: fc_chunk_decide_workspace_bytes(total elements, n_chunks) must not exceed the
  *     array, which holds 65,536 slab pairs: about 268 million elements over all chunks together,
  *     whatever the dtype.  Beyond it the call returns FC_ERR_TOO_LARGE and launches nothing.
- *   - The call never allocates or frees device memory.  The first call on each device looks up
- *     the array's device address (a driver query, made with that device current); make that
- *     first call before starting any stream capture.
+ *   - The call never allocates or frees device memory.  The array's device address is looked up
+ *     once per device (a driver query, made with that device current) by fc_create; should that
+ *     have failed, the first call on the device repeats it, so create the context, or make that
+ *     first call, before starting any stream capture.
  *   - All calls on a device share the one array, and it keeps the previous call's contents.
  *     Nothing in it has to start at zero (each slab pair is written before it is read), but two
  *     calls that overlap on the GPU (different streams, no dependency) race on it: serialise

@@ -17,6 +17,7 @@ struct fc_ctx {
 namespace fc {
 
 void set_cuda_error(cudaError_t e, const char* where);
+void decide_static_setup(int device);  // fc_decide.cu: address of the built-in scratch of fc_chunk_decide_static
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -53,6 +53,7 @@ extern "C" int fc_create(fc_ctx** out, int device) {
     delete ctx;
     return FC_ERR_CUDA;
   }
+  fc::decide_static_setup(device);
   *out = ctx;
   return FC_OK;
 }

@@ -288,7 +288,7 @@ constexpr int kMaxDevices = 64;
 // device address of g_decide_scratch on each device (null = not looked up yet)
 std::atomic<void*> g_scratch_addr[kMaxDevices];
 
-// Look the address up on first use per device.  Not an allocation: the array is part of the
+// Look the address up once per device (fc_create does it; the first call does if that did not happen).  Not an allocation: the array is part of the
 // module image every device already holds.  Concurrent first calls may both do the lookup; they
 // get the same answer and store the same value.
 int static_scratch(int device, void** out) {
@@ -313,6 +313,16 @@ int static_scratch(int device, void** out) {
 }
 
 }  // namespace
+
+namespace fc {
+// Called by fc_create with `device` current: looks the array's address up ahead of the first static call, so that
+// callers who may not touch the driver where they call do not pay for it there.  A failure here is not an error of
+// fc_create; the first fc_chunk_decide_static call then tries again and reports it.
+void decide_static_setup(int device) {
+  void* p = nullptr;
+  (void)static_scratch(device, &p);
+}
+}  // namespace fc
 
 extern "C" size_t fc_chunk_decide_static_max_bytes(void) { return kStaticScratchBytes; }
 

@@ -219,7 +219,13 @@ typedef struct {
  *                    between the decision and the attention.
  *   lse              DEVICE [H_q, lse_hs] fp32 or NULL: natural-log sum-exp of each computed row.
  * bf16 runs on tcgen05 tensor cores (fp32 accumulation in tensor memory, TMA-fed); fp32 runs
- * on CUDA cores with fp32 accumulation.  Workspace: fc_chunk_attention_workspace_bytes(). */
+ * on CUDA cores with fp32 accumulation.  With a token map the tensor-core kernel fetches K / V rows
+ * by index (four rows per copy instruction), at roughly three quarters of the segment-table rate;
+ * it needs K's and V's head strides to be whole numbers of rows, otherwise the CUDA-core kernel
+ * takes the call.  An index outside [0, kv_rows) sets FC_DEV_BAD_INDEX and is not followed.
+ * Physical rows that no visible logical token maps to (rows behind a segment's end, slots of
+ * the store that were never written) are never used, whatever they hold.
+ * Workspace: fc_chunk_attention_workspace_bytes(). */
 size_t fc_chunk_attention_workspace_bytes(const fc_attn_desc* desc);
 int fc_chunk_attention(fc_ctx* ctx, void* stream, const fc_attn_desc* desc, const void* Q,
                        const void* K, const void* V, int dtype, const int32_t* q_chunk_row_off,

@@ -116,7 +116,13 @@ extern "C" int fc_chunk_cache_apply(fc_ctx* ctx, void* stream, const void* x_in,
     if (slabs > INT32_MAX / 2) return FC_ERR_UNSUPPORTED;
   }
   if (chunk_elem_off[n_chunks] > 0 && (!x_in || !y_io || !cache)) return FC_ERR_INVALID_ARG;
-  if (x_in == y_io || x_in == cache || y_io == cache) return FC_ERR_INVALID_ARG;
+  {  // the three tensors must not overlap
+    const uintptr_t n = (uintptr_t)chunk_elem_off[n_chunks] * es;
+    const uintptr_t p[3] = {(uintptr_t)x_in, (uintptr_t)y_io, (uintptr_t)cache};
+    for (int a = 0; a < 3; ++a)
+      for (int b = a + 1; b < 3; ++b)
+        if (p[a] < p[b] + n && p[b] < p[a] + n) return FC_ERR_INVALID_ARG;
+  }
   if (slabs == 0) return FC_OK;
   cudaStream_t st = (cudaStream_t)stream;
   const unsigned grid = (unsigned)slabs;

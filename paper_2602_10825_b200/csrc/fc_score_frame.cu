@@ -31,10 +31,7 @@ using namespace fc::sm100;
 
 constexpr int kKeys = 128, kQueries = 128;  // tile: MMA M and N
 constexpr int kRing = 4;     // streamed tiles in flight = logit accumulators in tensor memory (4 x 128 columns)
-#ifndef FC_FRAME_FMA_SHARE
-#define FC_FRAME_FMA_SHARE 1
-#endif
-constexpr int kFmaShare = FC_FRAME_FMA_SHARE;  // of every four column pairs, how many take their exponential on the fma pipe
+constexpr int kFmaShare = 1;  // of every four column pairs, how many take their exponential on the fma pipe
 constexpr int kGroups = 4;   // consumer warpgroups; group g takes every fourth streamed tile
 constexpr int kThreads = 32 * (4 * kGroups + 2);  // 16 consumer warps, one copy warp, one MMA warp
 

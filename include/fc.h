@@ -11,6 +11,11 @@
  *   fc_kv_score           importance / redundancy score of cached tokens (Eqs. 9-12)
  *   fc_kv_select_compact  per-head top-B and retention of the chosen K/V rows
  *
+ * and a fifth for the step around the forward pass:
+ *
+ *   fc_chunk_cache_apply  chunks that were not recomputed are served from the
+ *                         activation cache (Sec. 3.2)
+ *
  * Conventions
  *   - Plain C types only.  Every pointer argument says whether it is a HOST or a
  *     DEVICE pointer.  The caller owns every buffer, including the workspace,

@@ -267,7 +267,8 @@ int fc_chunk_attention(fc_ctx* ctx, void* stream, const fc_attn_desc* desc, cons
 typedef enum { FC_RED_MEANKEY = 0, FC_RED_TILED = 1, FC_RED_TILED_MAX = 2 } fc_red_mode;
 
 typedef struct {
-  int32_t H_q, H_kv, d, L_q, L_k;  /* L_q * (H_q/H_kv) <= 128, or bf16 with H_q == H_kv and L_q <= 8192 */
+  int32_t H_q, H_kv, d, L_q, L_k;  /* n = L_q * (H_q/H_kv) queries per kv head: n <= 128, or bf16 with n <= 8192 and
+                                      either H_q == H_kv or the query heads stored one after the other (q_hs = L_q q_rs) */
   int64_t q_hs, q_rs, k_hs, k_rs;  /* element strides */
   float scale;                     /* 0 => 1/sqrt(d) */
   float lambda;                    /* mixing coefficient (paper: 0.07) */

@@ -3,8 +3,9 @@
 //
 // Two pipelines, both deterministic (no floating-point atomics).  bf16 inputs with one query head per key head
 // and at most 62 observation queries take the tensor-core kernels of fc_score_tc.cu followed by the finalize
-// kernel below; everything else (fp32, grouped query heads, more queries) takes the
-// CUDA-core pipeline (below).  bf16 inputs with more than 128 observation queries per key head (a latent frame
+// kernel below; everything else (fp32, more queries, grouped query heads whose rows are not contiguous) takes the
+// CUDA-core pipeline (below).  Grouped query heads stored head after head are folded into one head of group * L_q
+// queries first, so they take whichever pipeline that number of queries takes.  bf16 inputs with more than 128 observation queries per key head (a latent frame
 // or a whole chunk of them) take the frame-level pipeline: key norms and mean key by the CUDA-core pass-1 kernel
 // without queries, every query's log-sum-exp over the candidates and then the attention mass of every key by the
 // tensor-core kernel of fc_score_frame.cu (two launches), then the CUDA-core pass-2 kernel fed with that mass, and
@@ -313,12 +314,22 @@ int make_geom(const fc_score_desc* d, ScoreGeom& g) {
   if (d->pool_k < 1 || d->pool_k % 2 == 0) return FC_ERR_INVALID_ARG;
   if (d->d != 64 && d->d != 128) return FC_ERR_UNSUPPORTED;
   g.H_q = d->H_q; g.H_kv = d->H_kv; g.d = d->d; g.L_q = d->L_q; g.L_k = d->L_k;
+  g.q_hs = d->q_hs; g.q_rs = d->q_rs;
   g.group = d->H_q / d->H_kv;
-  g.n_q = g.group * d->L_q;
+  // Grouped query heads whose rows follow each other in memory (head stride = L_q rows) are one key head's worth of
+  // group * L_q observation queries: the importance is the mean over all of them (the group's heads and their rows)
+  // either way, and every pipeline, the tensor-core ones included, then sees one query head per key head.
+  if (g.group > 1 && d->q_hs == (int64_t)d->L_q * d->q_rs && (int64_t)g.group * d->L_q <= fc::kScoreFrameMaxQueries) {
+    g.L_q = g.group * d->L_q;
+    g.q_hs = (int64_t)g.group * d->q_hs;
+    g.H_q = d->H_kv;
+    g.group = 1;
+  }
+  g.n_q = g.group * g.L_q;
   if (g.n_q > kCoreMaxQueries && (g.group != 1 || g.L_q > fc::kScoreFrameMaxQueries)) return FC_ERR_UNSUPPORTED;
   g.n_tiles = (d->L_k + kTile - 1) / kTile;
   g.n_partials = g.n_tiles;
-  g.q_hs = d->q_hs; g.q_rs = d->q_rs; g.k_hs = d->k_hs; g.k_rs = d->k_rs;
+  g.k_hs = d->k_hs; g.k_rs = d->k_rs;
   g.scale = d->scale != 0.f ? d->scale : 1.f / sqrtf((float)d->d);
   g.lambda = d->lambda;
   g.pool_k = d->pool_k;

@@ -674,6 +674,24 @@ def test_score_gqa_and_d64(ctx):
     _score_case(ctx, Q, K, 0.2, 3)
 
 
+@pytest.mark.parametrize("g,L_q,L_k", [(2, 25, 1331), (4, 50, 2345), (8, 50, 900)])
+def test_score_grouped_query_heads_on_tensor_cores(ctx, g, L_q, L_k):
+    # grouped query heads, bf16: g heads x L_q rows per key head are g * L_q observation queries of that key head
+    # (50 -> the token-level tensor-core passes, 200 and 400 -> the frame-level ones); the importance is the mean over
+    # the group's heads and rows
+    H_kv = 2
+    Q = wl.normal((H_kv * g, L_q, 128), 91, 0.7, torch.bfloat16)
+    K = wl.normal((H_kv, L_k, 128), 92, 0.7, torch.bfloat16)
+    _score_case(ctx, Q, K, 0.07, 7)
+    # the same heads with a gap between them in memory are not one block of rows: the CUDA-core pipeline takes them
+    if g * L_q <= 128:
+        Qp = torch.zeros((H_kv * g, L_q + 3, 128), dtype=torch.bfloat16)
+        Qp[:, :L_q] = Q
+        want = oracle.kv_score(wl.bits(Q), wl.bits(K), lambda_=0.07, pool_k=7)
+        got = ctx.kv_score(dev(Qp)[:, :L_q], dev(K), lambda_=0.07, pool_k=7)["score"].double().cpu().numpy()
+        assert np.abs(got - want["score"]).max() <= 1e-4 * np.abs(want["score"]).max()
+
+
 def test_score_accumulated_over_steps(ctx):
     K = wl.normal((2, 700, 128), 41, 0.5, torch.bfloat16)
     Qs = [wl.normal((2, 50, 128), 42 + s, 0.5, torch.bfloat16) for s in range(3)]

@@ -56,7 +56,7 @@ using namespace fc::sm100;
 
 constexpr int kBM = 128, kBN = 128;
 constexpr int kHalf = kBN / 2;  // key columns per S accumulator
-constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {copy warp, two MMA warps, a spare warp}
+constexpr int kThreads = 384;  // 3 warpgroups: softmax A, softmax B, {copy warp, two MMA warps, the tail patcher}
 constexpr int kStages = 2;  // the MMA issuer computes stage and phase with masks: keep at 2
 constexpr uint32_t kTmemCols = 512;
 constexpr float kRescaleThreshold = 8.f;  // log2 units

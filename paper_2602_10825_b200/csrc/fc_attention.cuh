@@ -32,9 +32,9 @@ size_t attention_tc_workspace_bytes();
 int attention_ws_launch(fc_ctx* ctx, cudaStream_t st, const AttnGeom& g, const CUtensorMap& tq,
                         const CUtensorMap& tk, const CUtensorMap& tv, void* O, uint32_t* counter);
 bool attention_tc_supported(const AttnGeom& g, int dtype);
-// Tensor map of a [heads, rows, d] bf16 tensor: box = 64 elements (128 bytes) x 128 rows x 1 head, 128-byte
+// Tensor map of a [heads, rows, d] bf16 tensor: box = 64 elements (128 bytes) x `box_rows` rows x 1 head, 128-byte
 // swizzle; rows past `rows` read as zero.
 int make_tmap(fc_ctx* ctx, CUtensorMap* map, const void* base, int d, int64_t rows, int heads, int64_t row_stride,
-              int64_t head_stride);
+              int64_t head_stride, int box_rows = 128);
 
 }  // namespace fc

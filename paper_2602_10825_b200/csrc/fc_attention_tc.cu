@@ -18,10 +18,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 // [heads, rows, d] bf16 tensor, box = 64 elements (128 bytes) x 128 rows x 1 head, 128-byte swizzle.
 int make_tmap(fc_ctx* ctx, CUtensorMap* map, const void* base, int d, int64_t rows, int heads, int64_t row_stride,
-              int64_t head_stride) {
+              int64_t head_stride, int box_rows) {
   const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)heads};
   const cuuint64_t strides[2] = {(cuuint64_t)row_stride * 2, (cuuint64_t)head_stride * 2};
-  const cuuint32_t box[3] = {64, (cuuint32_t)kBM, 1};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = ((EncodeTiledFn)ctx->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base),
                                                   dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,

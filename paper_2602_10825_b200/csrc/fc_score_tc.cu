@@ -145,9 +145,14 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         for (int x = 0; x < kAtoms; ++x)
           tma_load_3d(smem_u32(k_tiles + st * kTileBytes + x * kAtomBytes), &tmap_k, bar, x * 64, tile_of(i) * kKeys, hk);
       };
-      mbar_expect_tx(smem_u32(&sh->q_full), kTileBytes);
+      // The query box is 64 rows high (at most 62 queries).  Pass 1 puts the queries into rows 0-63 AND rows 64-127
+      // of its A operand: the two logit warpgroups, which take alternate tiles, then read the same logits from
+      // different lane quadrants, i.e. with warps that sit on different schedulers (warps 0, 1 and warps 6, 7).
+      // With one copy, warps 0, 1 and 4, 5 did all the exponentials on two of the four schedulers.
+      mbar_expect_tx(smem_u32(&sh->q_full), PASS == 1 ? kTileBytes : kTileBytes / 2);
       for (int x = 0; x < kAtoms; ++x)
-        tma_load_3d(smem_u32(q_tile + x * kAtomBytes), &tmap_q, smem_u32(&sh->q_full), x * 64, 0, hk);
+        for (int rep = 0; rep < (PASS == 1 ? 2 : 1); ++rep)
+          tma_load_3d(smem_u32(q_tile + x * kAtomBytes + rep * 64 * 128), &tmap_q, smem_u32(&sh->q_full), x * 64, 0, hk);
       for (int i = 0; i < min(n, kRing - 1); ++i) load_k(i);
       mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
       if (PASS == 2) mbar_wait_bounded(smem_u32(&sh->q_patched), 0, abort);
@@ -180,9 +185,10 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     const uint32_t t_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     if (PASS == 1) {
       const int grp = warp >> 2;  // this warpgroup takes the tiles of its parity and the accumulator of that parity
-      const int q = tid & 127;    // query row
-      const bool row_ok = q < g.L_q;
-      const bool warp_ok = (warp & 3) * 32 < g.L_q;
+      const int q = (tid & 127) - grp * 64;  // query row: group 0 reads rows 0-63 of the accumulator, group 1 rows 64-127
+      const bool row_ok = q >= 0 && q < g.L_q;
+      const int q_warp = (warp & 3) * 32 - grp * 64;  // first query of this warp's lane quadrant
+      const bool warp_ok = q_warp >= 0 && q_warp < g.L_q;
       float m = -INFINITY, l = 0.f;
       for (int i = grp; i < n; i += 2) {
         const int b = grp;
@@ -233,7 +239,7 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         }
       }
       // the two warpgroups' results of the slice, merged in group order
-      if (grp == 1 && q < kNQ) sh->ml_s[q] = make_float2(m, l);
+      if (grp == 1 && q >= 0 && q < kNQ) sh->ml_s[q] = make_float2(m, l);
       asm volatile("bar.sync 4, 256;" ::: "memory");
       if (grp == 0 && row_ok) {
         const float2 p = sh->ml_s[q];
@@ -395,7 +401,7 @@ int score_tc_run(fc_ctx* ctx, cudaStream_t st, ScoreTcArgs g, int d, int64_t q_h
                  int64_t k_rs, const void* Q, const void* K) {
   CUtensorMap tq, tk;
   int rc;
-  if ((rc = make_tmap(ctx, &tq, Q, d, g.L_q, g.H, q_rs, g.H > 1 ? q_hs : q_rs * g.L_q)) != FC_OK) return rc;
+  if ((rc = make_tmap(ctx, &tq, Q, d, g.L_q, g.H, q_rs, g.H > 1 ? q_hs : q_rs * g.L_q, 64)) != FC_OK) return rc;
   if ((rc = make_tmap(ctx, &tk, K, d, g.L_k, g.H, k_rs, g.H > 1 ? k_hs : k_rs * g.L_k)) != FC_OK) return rc;
   // slices: one CTA per SM over all heads (a single wave), at most kScoreTcMaxSlices per head
   const int want = std::max(1, ctx->sm_count / g.H);

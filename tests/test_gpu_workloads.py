@@ -286,3 +286,86 @@ def test_streaming_generation_at_full_width(ctx):
         assert np.array_equal(wl.bits(sel["V_dst"].cpu()), want_sel["V_dst"])
         assert not np.array_equal(want_sel["kept_idx"][0], np.arange(B, dtype=np.int32))  # something was dropped
         hist_K, hist_V = sel["K_dst"].cpu(), sel["V_dst"].cpu()
+
+
+# ------------------------------------------------------------------------------------ the step as a CUDA graph
+
+def test_whole_step_replays_from_a_cuda_graph(ctx):
+    # No call allocates, synchronises or leaves its stream, and the work list never returns to the host, so one step
+    # (decide -> attention -> score -> select + compact -> cache apply) can be captured into a CUDA graph once and
+    # replayed on new data: the replay must give bit for bit what the same calls give when launched one by one, also
+    # when the new data changes which chunks are active.
+    w = wl.Workload("g", "bf16", H=4, d=128, W=3, n_c=333, B=211, L_k=544, seed=55, sigma=0.5, keys="clustered")
+    n_el = w.n_c * w.hidden
+    off = np.arange(w.W + 1, dtype=np.int64) * n_el
+    q_off, vis, slo, spo = wl.prefix_layout(w)
+    dev = "cuda"
+
+    def inputs(seed, targets):
+        cur, prev = wl.indicator_pair(w.W, n_el, targets, seed)
+        Q, K, V = wl.qkv(w, seed)
+        return dict(cur=cur, prev=prev, Q=Q, K=K, V=V)
+
+    first, second = inputs(1, [0.3, 0.01, 0.3]), inputs(2, [0.01, 0.3, 0.3])
+    st = {k: v.to(dev).clone() for k, v in first.items()}  # static input buffers of the graph
+    out = dict(acc=torch.zeros(w.W, device=dev), l1rel=torch.empty(w.W, device=dev),
+               recompute=torch.empty(w.W, dtype=torch.uint8, device=dev),
+               active_ids=torch.empty(w.W, dtype=torch.int32, device=dev), n_active=torch.empty(1, dtype=torch.int32, device=dev),
+               O=torch.zeros((w.H, w.window_rows, w.d), dtype=torch.bfloat16, device=dev),
+               score=torch.empty((w.H, w.L_k), device=dev), kept=torch.empty((w.H, w.B), dtype=torch.int32, device=dev),
+               n_kept=torch.empty(1, dtype=torch.int32, device=dev),
+               K_dst=torch.empty((w.H, w.B, w.d), dtype=torch.bfloat16, device=dev),
+               V_dst=torch.empty((w.H, w.B, w.d), dtype=torch.bfloat16, device=dev),
+               y=torch.zeros(w.W * n_el, dtype=torch.bfloat16, device=dev),
+               cache=torch.zeros(w.W * n_el, dtype=torch.bfloat16, device=dev),
+               status=torch.zeros(1, dtype=torch.int32, device=dev))
+    step_no = torch.full((w.W,), 4, dtype=torch.int32, device=dev)
+
+    def step():
+        ctx.chunk_decide(st["cur"], st["prev"], off, step_no, 1, 0.1, out["acc"], l1rel=out["l1rel"],
+                         recompute=out["recompute"], active_ids=out["active_ids"], n_active=out["n_active"], status=out["status"])
+        ctx.chunk_attention(st["Q"], st["K"], st["V"], q_off, vis, slo, spo, out["active_ids"], out["n_active"], out["O"],
+                            status=out["status"])
+        ctx.kv_score(st["Q"][:, -w.L_q_obs:], st["K"][:, :w.L_k], score=out["score"], status=out["status"])
+        ctx.kv_select_compact(out["score"], w.B, st["K"][:, :w.L_k], st["V"][:, :w.L_k], out["K_dst"], out["V_dst"],
+                              kept_idx=out["kept"], n_kept=out["n_kept"], status=out["status"])
+        ctx.chunk_cache_apply(st["cur"], out["y"], out["cache"], off, out["recompute"], status=out["status"])
+
+    def reset():
+        out["acc"].zero_(); out["O"].zero_(); out["y"].zero_(); out["cache"].zero_()
+
+    def snapshot():
+        return {k: v.clone() for k, v in out.items()}
+
+    # eager references for both data sets (this also sizes the binding's cached workspaces before the capture)
+    want = []
+    for data in (first, second):
+        for k, v in data.items():
+            st[k].copy_(v)
+        reset()
+        step()
+        torch.cuda.synchronize()
+        want.append(snapshot())
+    assert want[0]["recompute"].cpu().tolist() == [1, 0, 1] and want[1]["recompute"].cpu().tolist() == [0, 1, 1]
+    # capture once ...
+    for k, v in first.items():
+        st[k].copy_(v)
+    reset()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step()
+    torch.cuda.current_stream().wait_stream(side)
+    # ... replay on both data sets
+    for data, ref in ((first, want[0]), (second, want[1]), (first, want[0])):
+        for k, v in data.items():
+            st[k].copy_(v)
+        reset()
+        graph.replay()
+        torch.cuda.synchronize()
+        for k in out:
+            assert torch.equal(out[k].view(torch.uint8) if out[k].dtype == torch.bfloat16 else out[k],
+                               ref[k].view(torch.uint8) if ref[k].dtype == torch.bfloat16 else ref[k]), k
+    assert out["status"].item() == 0

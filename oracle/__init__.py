@@ -241,3 +241,19 @@ def kv_select_compact(score, B, K_src=None, V_src=None, n_threads=0):
     if rc:
         raise ValueError(f"fco_kv_select_compact -> {rc}")
     return dict(kept_idx=kept, n_kept=int(cnt[0]), K_dst=K_dst, V_dst=V_dst)
+
+
+def kv_select_units(score, B, unit=1, n_protect=0, n_threads=0):
+    """Selection by units of ``unit`` consecutive tokens (unit score = mean of the tokens' scores) with the last
+    ``n_protect`` tokens' units always kept.  Returns dict(kept_idx [H, min(B, L_k)] ascending, n_kept)."""
+    score = np.ascontiguousarray(score, dtype=np.float32)
+    H, L_k = score.shape
+    n_keep = min(B, L_k)
+    kept = np.zeros((H, n_keep), np.int32)
+    cnt = np.zeros(1, np.int32)
+    rc = lib().fco_kv_select_units(_ptr(score), H, L_k, int(B), int(unit), int(n_protect), _ptr(kept), _ptr(cnt),
+                                   int(n_threads))
+    if rc:
+        raise ValueError(f"fco_kv_select_units -> {rc}")
+    return dict(kept_idx=kept, n_kept=int(cnt[0]))
+

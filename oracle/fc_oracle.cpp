@@ -559,3 +559,48 @@ extern "C" int fco_kv_select_compact(const float* score, int n_heads, int L_k,
   });
   return 0;
 }
+
+// ---------------------------------------------------------------------------
+// Selection at a coarser key granularity (the key-granularity ablation of the
+// paper's Table 4: frame- or chunk-level keys instead of tokens) and with a
+// protected tail.  Units of `unit` consecutive tokens are kept or dropped as a
+// whole; a unit's score is the mean of its tokens' scores (fp64 sum in token
+// order, rounded to fp32: the selection compares fp32 values as the token-level
+// one does).  The last ceil(n_protect / unit) units (the newest tokens) are kept
+// whatever their score.  Order among the others: score descending, unit index
+// ascending, NaN as -inf.  kept_idx lists the tokens of the kept units ascending.
+// ---------------------------------------------------------------------------
+extern "C" int fco_kv_select_units(const float* score, int n_heads, int L_k, int B, int unit,
+                                   int n_protect, int32_t* kept_idx, int32_t* n_kept,
+                                   int n_threads) {
+  if (!score || !kept_idx || n_heads <= 0 || L_k <= 0 || B <= 0 || unit <= 0 || n_protect < 0) return -1;
+  if (L_k % unit || B % unit) return -2;
+  const int n_units = L_k / unit, keep_units = std::min(B / unit, n_units);
+  const int protect_units = std::min((n_protect + unit - 1) / unit, keep_units);
+  if (n_kept) *n_kept = keep_units * unit;
+  parallel_for(n_heads, n_threads, [&](int64_t h) {
+    const float* s = score + h * L_k;
+    std::vector<float> us(n_units);
+    for (int u = 0; u < n_units; ++u) {
+      double acc = 0.0;
+      for (int t = 0; t < unit; ++t) acc += (double)s[(int64_t)u * unit + t];
+      us[u] = (float)(acc / (double)unit);
+    }
+    auto rank_value = [&](int u) {
+      return std::isnan(us[u]) ? -std::numeric_limits<float>::infinity() : us[u];
+    };
+    std::vector<int32_t> order(n_units - protect_units);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+      return rank_value(a) > rank_value(b);  // stable => index ascending on ties
+    });
+    std::vector<int32_t> kept(order.begin(), order.begin() + (keep_units - protect_units));
+    for (int u = n_units - protect_units; u < n_units; ++u) kept.push_back(u);
+    std::sort(kept.begin(), kept.end());
+    for (int r = 0; r < keep_units; ++r)
+      for (int t = 0; t < unit; ++t)
+        kept_idx[h * (int64_t)keep_units * unit + (int64_t)r * unit + t] = kept[r] * unit + t;
+  });
+  return 0;
+}
+

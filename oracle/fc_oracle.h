@@ -153,6 +153,17 @@ int fco_kv_select_compact(const float* score, int n_heads, int L_k, int B,
 
 int fco_hardware_threads(void);
 
+/* Selection at a coarser key granularity (key-granularity ablation, Table 4) and
+ * with a protected tail: units of `unit` consecutive tokens (L_k and B multiples
+ * of it) are kept or dropped as a whole; unit score = mean of its tokens' scores
+ * (fp64 sum, rounded to fp32); the last ceil(n_protect / unit) units are always
+ * kept; the others rank by (score desc, index asc), NaN as -inf.  kept_idx
+ * [n_heads, min(B, L_k)] lists the kept tokens ascending.  unit = 1 and
+ * n_protect = 0 is the selection of fco_kv_select_compact. */
+int fco_kv_select_units(const float* score, int n_heads, int L_k, int B, int unit,
+                        int n_protect, int32_t* kept_idx, int32_t* n_kept,
+                        int n_threads);
+
 #ifdef __cplusplus
 }
 #endif

@@ -528,3 +528,41 @@ def test_similarity_columns_match_the_full_matrix_and_the_mean_key_identity():
     for mode in (oracle.RED_PLAIN, oracle.RED_MEANKEY):
         red = oracle.kv_score(wl.bits(Q), wl.bits(K), red_mode=mode)["red"]
         np.testing.assert_allclose(red, torch.softmax(torch.from_numpy(full), dim=-1).numpy(), rtol=1e-10)
+
+
+# --------------------------------------------------------------------------- selection by units, protected tail
+
+def test_select_units_hand_example(golden):
+    g = golden("select_units_hand_example.txt")
+    score = np.array([g["score"]], np.float32)
+    for n_protect, key in ((0, "kept_p0"), (2, "kept_p2"), (4, "kept_p4")):
+        out = oracle.kv_select_units(score, 6, unit=3, n_protect=n_protect)
+        assert out["kept_idx"][0].tolist() == [int(v) for v in g[key]] and out["n_kept"] == 6
+
+
+def test_select_units_reduce_to_the_token_level_selection_and_match_a_library_topk():
+    rng = np.random.default_rng(17)
+    score = rng.normal(size=(3, 240)).astype(np.float32)
+    score[0, ::7] = score[0, 3]   # ties
+    score[1, 11] = np.nan
+    # unit 1, nothing protected: exactly the token-level selection
+    for B in (1, 17, 239, 240, 300):
+        a = oracle.kv_select_units(score, B)["kept_idx"]
+        b = oracle.kv_select_compact(score, B)["kept_idx"]
+        assert np.array_equal(a, b)
+    # units of 8: torch's mean (fp64) and topk on distinct unit means
+    s = torch.from_numpy(np.ascontiguousarray(score[2:])).double()
+    means = s.reshape(1, 30, 8).mean(-1).float()
+    want_units = torch.sort(torch.topk(means, 12, dim=1).indices, dim=1).values
+    want = (want_units[:, :, None] * 8 + torch.arange(8)).reshape(1, -1).numpy()
+    got = oracle.kv_select_units(np.ascontiguousarray(score[2:]), 96, unit=8)
+    assert np.array_equal(got["kept_idx"], want) and got["n_kept"] == 96
+    # a protected tail at token level: the last 5 tokens plus the best 12 of the others
+    got = oracle.kv_select_units(np.ascontiguousarray(score[2:]), 17, n_protect=5)["kept_idx"][0]
+    rest = np.sort(np.argsort(-score[2, :235], kind="stable")[:12])
+    assert got.tolist() == rest.tolist() + [235, 236, 237, 238, 239]
+    # budget at least the cache length: identity; protection beyond the budget is capped by it
+    assert oracle.kv_select_units(score, 240, unit=8)["kept_idx"][0].tolist() == list(range(240))
+    assert oracle.kv_select_units(score, 16, unit=8, n_protect=100)["kept_idx"][0].tolist() == list(range(224, 240))
+    with pytest.raises(ValueError):
+        oracle.kv_select_units(score, 100, unit=8)  # the budget must be a whole number of units

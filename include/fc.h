@@ -317,6 +317,27 @@ int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* score, int n_he
                          int dtype, int d, const fc_compact_strides* strides, int32_t* kept_idx,
                          int32_t* n_kept, uint32_t* status, void* ws, size_t ws_bytes);
 
+/* fc_kv_select_compact_ex — the same selection at a coarser key granularity and / or with a protected tail.
+ *
+ * Paper: the key-granularity ablation (Table 4) compresses with frame- or chunk-level keys instead of tokens (and
+ * finds token-level keys best, which is why fc_kv_select_compact is the default).  Here a unit is `unit`
+ * consecutive tokens (a latent frame, a chunk), kept or dropped as a whole; a unit's score is the mean of its
+ * tokens' scores (fp64 sum, rounded to fp32); L_k and B must be whole numbers of units.  n_protect (not in the
+ * paper) keeps the units of the last n_protect tokens - the newest ones - whatever their score; the others rank
+ * by (score descending, index ascending), NaN as -inf.  unit = 1, n_protect = 0 is fc_kv_select_compact.
+ * Workspace (only for unit > 1): fc_kv_select_compact_ex_workspace_bytes().  All other arguments as above;
+ * kept_idx lists the kept tokens ascending, n_kept = min(B, L_k). */
+typedef struct {
+  int32_t unit;      /* tokens per selection unit, >= 1 */
+  int32_t n_protect; /* newest tokens always kept, >= 0 */
+} fc_select_opts;
+
+size_t fc_kv_select_compact_ex_workspace_bytes(int n_heads, int L_k, int unit);
+int fc_kv_select_compact_ex(fc_ctx* ctx, void* stream, const float* score, int n_heads, int L_k, int B,
+                            const fc_select_opts* opts, const void* K_src, const void* V_src, void* K_dst,
+                            void* V_dst, int dtype, int d, const fc_compact_strides* strides, int32_t* kept_idx,
+                            int32_t* n_kept, uint32_t* status, void* ws, size_t ws_bytes);
+
 #ifdef __cplusplus
 }
 #endif

@@ -38,6 +38,10 @@ class _ScoreDesc(C.Structure):
                 ("pool_k", C.c_int32), ("impl", C.c_int32), ("red_mode", C.c_int32)]
 
 
+class _SelectOpts(C.Structure):
+    _fields_ = [("unit", C.c_int32), ("n_protect", C.c_int32)]
+
+
 class _CompactStrides(C.Structure):
     _fields_ = [("src_hs", C.c_int64), ("src_rs", C.c_int64), ("dst_hs", C.c_int64), ("dst_rs", C.c_int64)]
 
@@ -60,7 +64,8 @@ def lib():
         L.fc_status_string.restype = C.c_char_p
         L.fc_last_cuda_error.restype = C.c_char_p
         for name in ("fc_chunk_decide_static_max_bytes", "fc_chunk_decide_workspace_bytes", "fc_chunk_attention_workspace_bytes",
-                     "fc_kv_score_workspace_bytes", "fc_kv_select_compact_workspace_bytes"):
+                     "fc_kv_score_workspace_bytes", "fc_kv_select_compact_workspace_bytes",
+                     "fc_kv_select_compact_ex_workspace_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.fc_chunk_decide_workspace_bytes.argtypes = [C.c_int64, C.c_int]
         _lib = L
@@ -279,7 +284,8 @@ class Context:
 
     # ------------------------------------------------------------------ fc_kv_select_compact
     def kv_select_compact(self, score, B, K_src=None, V_src=None, K_dst=None, V_dst=None, *, kept_idx=None,
-                          n_kept=None, status=None, ws=None):
+                          n_kept=None, status=None, ws=None, unit=1, n_protect=0):
+        """fc_kv_select_compact, or fc_kv_select_compact_ex when a selection unit or a protected tail is given."""
         H, L_k = score.shape
         if not score.is_contiguous():
             raise FcError("score must be contiguous [n_heads, L_k]")
@@ -300,6 +306,18 @@ class Context:
                 raise FcError("K_dst and V_dst must share strides")
             strides = _CompactStrides(s_hs, s_rs, d_hs, d_rs)
             dtype, d = _dt(K_src), K_src.shape[2]
+        if unit != 1 or n_protect != 0:
+            need = self._L.fc_kv_select_compact_ex_workspace_bytes(H, L_k, int(unit))
+            ws = self.workspace("select", need) if ws is None else ws
+            opts = _SelectOpts(int(unit), int(n_protect))
+            rc = self._L.fc_kv_select_compact_ex(
+                self._h, self._stream(), _dev(score, "score", torch.float32), H, L_k, int(B), C.byref(opts),
+                _dev(K_src, "K_src"), _dev(V_src, "V_src"), _dev(K_dst, "K_dst"), _dev(V_dst, "V_dst"), dtype, d,
+                None if strides is None else C.byref(strides), _dev(kept_idx, "kept_idx", torch.int32),
+                _dev(n_kept, "n_kept", torch.int32), _dev(status, "status", torch.int32), _dev(ws, "ws"),
+                C.c_size_t(ws.numel()))
+            self._check(rc, "fc_kv_select_compact_ex")
+            return dict(kept_idx=kept_idx, n_kept=n_kept, K_dst=K_dst, V_dst=V_dst)
         need = self._L.fc_kv_select_compact_workspace_bytes(H, L_k)
         ws = self.workspace("select", need) if ws is None else ws
         rc = self._L.fc_kv_select_compact(

@@ -13,6 +13,8 @@
 // independent loads in flight per thread; rows that were dropped are never read.  It is launched as a programmatic
 // dependent of the selection: its blocks take their places on the SMs while the selection still runs and start
 // copying the moment it has ended.
+#include <algorithm>
+
 #include <cooperative_groups.h>
 
 #include "fc_common.cuh"
@@ -47,8 +49,8 @@ struct SelShared {
 
 template <bool kSmemKeys>
 __global__ void __launch_bounds__(kSelThreads)
-select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, int32_t* __restrict__ kept_idx,
-                   int32_t* __restrict__ n_kept, uint32_t* __restrict__ status) {
+select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, int protect_from,
+                   int32_t* __restrict__ kept_idx, int32_t* __restrict__ n_kept, uint32_t* __restrict__ status) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ uint32_t smem_keys[];
@@ -83,8 +85,9 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
       const int j = j0 + u * kSelThreads;
       if (j < n) {
         bool nn;
-        const uint32_t k = score_key(v[u], nn);
+        uint32_t k = score_key(v[u], nn);
         any_nan |= nn;
+        if (begin + j >= protect_from) k = 0xffffffffu;  // protected tail: above every score's key (+inf is 0xff800000)
         if (kSmemKeys) smem_keys[j] = k;
         kmin = min(kmin, k);
         kmax = max(kmax, k);
@@ -127,7 +130,7 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
   auto key_at = [&](int j) -> uint32_t {  // key relative to the head's minimum; j is local to this CTA
     if (kSmemKeys) return smem_keys[j] - base;
     bool nn;
-    return score_key(s[j], nn) - base;
+    return (begin + j >= protect_from ? 0xffffffffu : score_key(s[j], nn)) - base;
   };
 
   // Radix select, most significant digit first, kDigitBits at a time over the n_bits that vary.  Invariant: the
@@ -321,6 +324,111 @@ gather_rows_kernel(const uint8_t* __restrict__ K_src, const uint8_t* __restrict_
 }
 
 
+// Selection units (a latent frame, a chunk): mean score of the `unit` consecutive tokens of every unit.  One warp per
+// unit: each lane adds every 32nd score in fp64, the lanes are combined in a fixed tree; fp64 sums of fp32 scores of
+// one head are exact for any realistic spread of magnitudes, so the order of summation does not show in the result.
+__global__ void __launch_bounds__(256)
+unit_mean_kernel(const float* __restrict__ score, int L_k, int unit, int n_units, int n_heads,
+                 float* __restrict__ unit_score) {
+  const int w = (int)((blockIdx.x * 256 + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+  if (w >= n_heads * n_units) return;
+  const int h = w / n_units, u = w % n_units;
+  const float* s = score + (size_t)h * L_k + (size_t)u * unit;
+  double acc = 0.0;
+  for (int t = lane; t < unit; t += 32) acc += (double)s[t];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, o);
+  if (lane == 0) unit_score[w] = (float)(acc / (double)unit);
+}
+
+// kept units -> kept tokens (ascending, as the units are)
+__global__ void expand_units_kernel(const int32_t* __restrict__ unit_idx, int keep_units, int unit, int n_heads,
+                                    int32_t* __restrict__ kept_idx, int32_t* __restrict__ n_kept) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t per_head = (int64_t)keep_units * unit;
+  if (i == 0 && n_kept) *n_kept = (int32_t)per_head;
+  if (i >= per_head * n_heads) return;
+  const int h = (int)(i / per_head), r = (int)((i % per_head) / unit), t = (int)(i % unit);
+  kept_idx[i] = unit_idx[(size_t)h * keep_units + r] * unit + t;
+}
+
+// Top-B of [n_heads, L] scores into out_idx [n_heads, min(B, L)]; entries at or after `protect_from` are kept first.
+int launch_select(fc_ctx* ctx, cudaStream_t st, const float* score, int n_heads, int L, int B, int protect_from,
+                  int32_t* out_idx, int32_t* n_kept, uint32_t* status) {
+  if (B >= L) {
+    const int64_t n = (int64_t)n_heads * L;
+    select_identity_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(out_idx, n_heads, L, score, n_kept, status);
+    FC_LAUNCH_CHECK("select_identity_kernel");
+    return FC_OK;
+  }
+  // cluster size: as many CTAs per head as keep all heads within one wave of the SMs
+  int cs = 1;
+  while (cs < kMaxCluster && n_heads * cs * 2 <= ctx->sm_count) cs *= 2;
+  const int chunk = (L + cs - 1) / cs;
+  const size_t key_bytes = (size_t)chunk * 4;
+  const bool smem_keys = key_bytes + sizeof(SelShared) + 1024 <= (size_t)ctx->smem_optin;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)n_heads * cs);
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = smem_keys ? key_bytes : 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cs;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may be scheduled under the previous kernel's tail
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  if (smem_keys) {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+    FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<true>, score, L, B, chunk, protect_from, out_idx, n_kept, status));
+  } else {
+    FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<false>, score, L, B, chunk, protect_from, out_idx, n_kept, status));
+  }
+  FC_LAUNCH_CHECK("select_topb_kernel");
+  return FC_OK;
+}
+
+struct CopyArgs {
+  const void *K_src, *V_src;
+  void *K_dst, *V_dst;
+  int dtype, d;
+  const fc_compact_strides* strides;
+};
+
+int check_copy(const CopyArgs& c, bool& copy) {
+  copy = c.K_src || c.V_src || c.K_dst || c.V_dst;
+  if (!copy) return FC_OK;
+  if (!c.K_src || !c.V_src || !c.K_dst || !c.V_dst || !c.strides) return FC_ERR_INVALID_ARG;
+  if (c.dtype != FC_BF16 && c.dtype != FC_F32) return FC_ERR_UNSUPPORTED;
+  if (c.d <= 0) return FC_ERR_INVALID_ARG;
+  const int es = fc::elem_size(c.dtype);
+  if ((c.d * es) % 16) return FC_ERR_UNSUPPORTED;
+  if (!fc::aligned16(c.K_src) || !fc::aligned16(c.V_src) || !fc::aligned16(c.K_dst) || !fc::aligned16(c.V_dst))
+    return FC_ERR_MISALIGNED;
+  const int64_t st[4] = {c.strides->src_hs, c.strides->src_rs, c.strides->dst_hs, c.strides->dst_rs};
+  for (int i = 0; i < 4; ++i)
+    if (st[i] < 0 || (st[i] * es) % 16) return FC_ERR_MISALIGNED;
+  if (c.strides->src_rs < c.d || c.strides->dst_rs < c.d) return FC_ERR_INVALID_ARG;
+  return FC_OK;
+}
+
+int launch_gather(cudaStream_t st, const CopyArgs& c, const int32_t* kept_idx, int n_heads, int n_keep, int L_k,
+                  uint32_t* status) {
+  const int es = fc::elem_size(c.dtype);
+  const int ppr = c.d * es / 16;
+  const int64_t n_pieces = (int64_t)n_keep * ppr;
+  dim3 grid((unsigned)((n_pieces + kCopyThreads * kUnroll - 1) / (kCopyThreads * kUnroll)), n_heads);
+  FC_CUDA_CHECK(fc::launch_pdl(gather_rows_kernel, grid, dim3(kCopyThreads), 0, st, (const uint8_t*)c.K_src,
+                               (const uint8_t*)c.V_src, (uint8_t*)c.K_dst, (uint8_t*)c.V_dst, kept_idx, n_keep, L_k, ppr,
+                               c.strides->src_hs * es, c.strides->src_rs * es, c.strides->dst_hs * es,
+                               c.strides->dst_rs * es, status));
+  FC_LAUNCH_CHECK("gather_rows_kernel");
+  return FC_OK;
+}
+
 }  // namespace
 
 extern "C" size_t fc_kv_select_compact_workspace_bytes(int n_heads, int L_k) {
@@ -336,67 +444,58 @@ extern "C" int fc_kv_select_compact(fc_ctx* ctx, void* stream, const float* scor
   (void)ws;
   (void)ws_bytes;
   if (!ctx || !score || !kept_idx || n_heads <= 0 || L_k <= 0 || B <= 0) return FC_ERR_INVALID_ARG;
-  const bool copy = K_src || V_src || K_dst || V_dst;
-  if (copy) {
-    if (!K_src || !V_src || !K_dst || !V_dst || !strides) return FC_ERR_INVALID_ARG;
-    if (dtype != FC_BF16 && dtype != FC_F32) return FC_ERR_UNSUPPORTED;
-    if (d <= 0) return FC_ERR_INVALID_ARG;
-    const int es = fc::elem_size(dtype);
-    if ((d * es) % 16) return FC_ERR_UNSUPPORTED;
-    if (!fc::aligned16(K_src) || !fc::aligned16(V_src) || !fc::aligned16(K_dst) || !fc::aligned16(V_dst))
-      return FC_ERR_MISALIGNED;
-    const int64_t st[4] = {strides->src_hs, strides->src_rs, strides->dst_hs, strides->dst_rs};
-    for (int i = 0; i < 4; ++i)
-      if (st[i] < 0 || (st[i] * es) % 16) return FC_ERR_MISALIGNED;
-    if (strides->src_rs < d || strides->dst_rs < d) return FC_ERR_INVALID_ARG;
-  }
+  const CopyArgs c = {K_src, V_src, K_dst, V_dst, dtype, d, strides};
+  bool copy;
+  int rc = check_copy(c, copy);
+  if (rc != FC_OK) return rc;
   if (L_k > (1 << 20)) return FC_ERR_UNSUPPORTED;  // keeps the packed 16-bit scan counters exact
   cudaStream_t st = (cudaStream_t)stream;
+  if ((rc = launch_select(ctx, st, score, n_heads, L_k, B, L_k, kept_idx, n_kept, status)) != FC_OK) return rc;
+  if (copy) return launch_gather(st, c, kept_idx, n_heads, B < L_k ? B : L_k, L_k, status);
+  return FC_OK;
+}
+
+extern "C" size_t fc_kv_select_compact_ex_workspace_bytes(int n_heads, int L_k, int unit) {
+  if (n_heads <= 0 || L_k <= 0 || unit <= 1) return 16;
+  const size_t n_units = (size_t)(L_k / unit);
+  return fc::align_up(n_heads * n_units * sizeof(float), 256) + fc::align_up(n_heads * n_units * sizeof(int32_t), 256);
+}
+
+extern "C" int fc_kv_select_compact_ex(fc_ctx* ctx, void* stream, const float* score, int n_heads, int L_k, int B,
+                                       const fc_select_opts* opts, const void* K_src, const void* V_src, void* K_dst,
+                                       void* V_dst, int dtype, int d, const fc_compact_strides* strides,
+                                       int32_t* kept_idx, int32_t* n_kept, uint32_t* status, void* ws, size_t ws_bytes) {
+  if (!ctx || !score || !kept_idx || !opts || n_heads <= 0 || L_k <= 0 || B <= 0) return FC_ERR_INVALID_ARG;
+  const int unit = opts->unit, n_protect = opts->n_protect;
+  if (unit <= 0 || n_protect < 0) return FC_ERR_INVALID_ARG;
+  if (L_k % unit || B % unit) return FC_ERR_INVALID_ARG;  // whole units only
+  const CopyArgs c = {K_src, V_src, K_dst, V_dst, dtype, d, strides};
+  bool copy;
+  int rc = check_copy(c, copy);
+  if (rc != FC_OK) return rc;
+  if (L_k > (1 << 20)) return FC_ERR_UNSUPPORTED;
+  cudaStream_t st = (cudaStream_t)stream;
   const int n_keep = B < L_k ? B : L_k;
-  if (B >= L_k) {
-    const int64_t n = (int64_t)n_heads * L_k;
-    select_identity_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(kept_idx, n_heads, L_k, score, n_kept, status);
-    FC_LAUNCH_CHECK("select_identity_kernel");
+  if (unit == 1) {
+    const int protect = n_protect < n_keep ? n_protect : n_keep;
+    if ((rc = launch_select(ctx, st, score, n_heads, L_k, B, L_k - protect, kept_idx, n_kept, status)) != FC_OK) return rc;
   } else {
-    // cluster size: as many CTAs per head as keep all heads within one wave of the SMs
-    int cs = 1;
-    while (cs < kMaxCluster && n_heads * cs * 2 <= ctx->sm_count) cs *= 2;
-    const int chunk = (L_k + cs - 1) / cs;
-    const size_t key_bytes = (size_t)chunk * 4;
-    const bool smem_keys = key_bytes + sizeof(SelShared) + 1024 <= (size_t)ctx->smem_optin;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)n_heads * cs);
-    cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = smem_keys ? key_bytes : 0;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = cs;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may be scheduled under the previous kernel's tail
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
-    if (smem_keys) {
-      FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>,
-                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
-      FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<true>, score, L_k, B, chunk, kept_idx, n_kept, status));
-    } else {
-      FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<false>, score, L_k, B, chunk, kept_idx, n_kept, status));
-    }
-    FC_LAUNCH_CHECK("select_topb_kernel");
+    const int n_units = L_k / unit, keep_units = n_keep / unit;
+    const int protect_units = std::min((n_protect + unit - 1) / unit, keep_units);
+    if (!ws || ws_bytes < fc_kv_select_compact_ex_workspace_bytes(n_heads, L_k, unit)) return FC_ERR_WORKSPACE;
+    if (!fc::aligned16(ws)) return FC_ERR_MISALIGNED;
+    float* unit_score = (float*)ws;
+    int32_t* unit_idx = (int32_t*)((char*)ws + fc::align_up((size_t)n_heads * n_units * sizeof(float), 256));
+    const int64_t warps = (int64_t)n_heads * n_units;
+    unit_mean_kernel<<<(unsigned)((warps * 32 + 255) / 256), 256, 0, st>>>(score, L_k, unit, n_units, n_heads, unit_score);
+    FC_LAUNCH_CHECK("unit_mean_kernel");
+    if ((rc = launch_select(ctx, st, unit_score, n_heads, n_units, keep_units, n_units - protect_units, unit_idx, nullptr,
+                            status)) != FC_OK)
+      return rc;
+    const int64_t n = (int64_t)n_heads * keep_units * unit;
+    expand_units_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(unit_idx, keep_units, unit, n_heads, kept_idx, n_kept);
+    FC_LAUNCH_CHECK("expand_units_kernel");
   }
-  if (copy) {
-    const int es = fc::elem_size(dtype);
-    const int ppr = d * es / 16;
-    const int64_t n_pieces = (int64_t)n_keep * ppr;
-    dim3 grid((unsigned)((n_pieces + kCopyThreads * kUnroll - 1) / (kCopyThreads * kUnroll)), n_heads);
-    FC_CUDA_CHECK(fc::launch_pdl(gather_rows_kernel, grid, dim3(kCopyThreads), 0, st, (const uint8_t*)K_src,
-                                 (const uint8_t*)V_src, (uint8_t*)K_dst, (uint8_t*)V_dst, (const int32_t*)kept_idx, n_keep,
-                                 L_k, ppr, strides->src_hs * es, strides->src_rs * es, strides->dst_hs * es,
-                                 strides->dst_rs * es, status));
-    FC_LAUNCH_CHECK("gather_rows_kernel");
-  }
+  if (copy) return launch_gather(st, c, kept_idx, n_heads, n_keep, L_k, status);
   return FC_OK;
 }

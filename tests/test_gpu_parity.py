@@ -800,6 +800,52 @@ def test_select_large_head_falls_back_to_global_keys(ctx):
     _select_case(ctx, score, 33333)
 
 
+def _select_units_case(ctx, score, B, unit, n_protect, K=None, V=None):
+    want = oracle.kv_select_units(score, B, unit=unit, n_protect=n_protect)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    got = ctx.kv_select_compact(torch.from_numpy(score).cuda(), B, None if K is None else dev(K),
+                                None if V is None else dev(V), status=status, unit=unit, n_protect=n_protect)
+    torch.cuda.synchronize()
+    kept = got["kept_idx"].cpu().numpy()
+    assert np.array_equal(kept, want["kept_idx"]), (B, unit, n_protect)
+    assert int(got["n_kept"].item()) == want["n_kept"]
+    if K is not None:  # the rows of the kept tokens, byte for byte
+        idx = torch.from_numpy(kept.astype(np.int64))[:, :, None].expand(-1, -1, K.shape[2])
+        assert np.array_equal(wl.bits(got["K_dst"].cpu()), wl.bits(torch.gather(K, 1, idx)))
+        assert np.array_equal(wl.bits(got["V_dst"].cpu()), wl.bits(torch.gather(V, 1, idx)))
+    return status.item()
+
+
+def test_select_by_units_and_with_a_protected_tail(ctx):
+    rng = np.random.default_rng(23)
+    score = rng.normal(size=(4, 4800)).astype(np.float32)
+    score[:, ::5] = score[:, 2:3]      # many equal scores
+    score[1, 17] = np.nan
+    score[3] = 1.0                      # a head where everything ties
+    # token level with the newest tokens protected (also more protected tokens than the budget holds)
+    for B, n_protect in ((1000, 1), (1000, 300), (2500, 2500), (64, 500), (4800, 10)):
+        st = _select_units_case(ctx, score, B, 1, n_protect)
+        assert st & 2 or B >= 4800  # the NaN was reported (the identity path reports it too)
+    # units of 8, 100 and 1600 tokens (a NaN makes its whole unit rank last), with and without protection
+    for unit, B, n_protect in ((8, 2400, 0), (8, 2400, 20), (100, 1200, 0), (100, 4800, 0), (1600, 3200, 1), (1600, 1600, 0)):
+        _select_units_case(ctx, score, B, unit, n_protect)
+    import paper_2602_10825_b200 as fc
+    with pytest.raises(fc.FcError, match="invalid"):   # whole units only
+        ctx.kv_select_compact(torch.from_numpy(score).cuda(), 1000, unit=7)
+
+
+@pytest.mark.parametrize("name", ["cached_step_bf16", "sweep_bf16"])
+def test_select_by_latent_frames_at_full_size(ctx, name):
+    # the key-granularity ablation at the benchmark's sizes: units of one latent frame (30 x 52 = 1560 tokens), scores
+    # from the library itself fed to both sides, kept frames bit-exact, compacted rows byte-exact
+    w = wl.CONFIGS[name]
+    Q_obs, K, V = wl.candidates(w)
+    score = ctx.kv_score(dev(Q_obs), dev(K), lambda_=w.lam, pool_k=w.pool_k)["score"].cpu().numpy()
+    assert w.L_k % 1560 == 0 and w.B % 1560 == 0
+    _select_units_case(ctx, score, w.B, 1560, 0, K, V)
+    _select_units_case(ctx, score, w.B, 1560, 1560, K, V)   # the newest frame protected
+
+
 def test_pipeline_gpu_scores_feed_gpu_select(ctx):
     # end to end on the device: score -> select on the library's own fp32 scores; the oracle's
     # selection on those same scores (copied back) must give the same indices

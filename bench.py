@@ -18,6 +18,7 @@ With --impl reference the oracle itself is the timed program (host cores only).
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import hashlib
 import json
 import os
@@ -576,10 +577,13 @@ def time_token_map_attention(step, iters=5):
     return time_calls(fn, iters, 2)
 
 
-def time_single_step_attention(ctx, device, iters=20):
+def time_single_step_attention(ctx, device, iters=20, head_dim=128):
     """The attention kernel alone on the single-step configuration (16 heads, 4 x 6240 tokens, no clean region):
-    short enough to run at burst clocks.  Returns (ms, algorithmic FLOPs)."""
+    short enough to run at burst clocks.  head_dim = 64: the same hidden width as 32 heads of 64.
+    Returns (ms, algorithmic FLOPs)."""
     w = wl.CONFIGS["single_step_bf16"]
+    if head_dim != w.d:
+        w = dataclasses.replace(w, name=f"{w.name}_d{head_dim}", H=w.H * w.d // head_dim, d=head_dim)
     st = DeviceStep(ctx, w, seed=0, device=device, attention_only=True)
     st.n_active.fill_(w.W)
     st.active_ids.copy_(torch.arange(w.W, dtype=torch.int32, device=device))
@@ -634,9 +638,10 @@ def main():
         fc_build.build()
     barrier()
     ctx = fc.Context(local_rank)
-    single = None
+    single = single_d64 = None
     if world == 1 and w.dtype == "bf16" and w.name != "single_step_bf16" and not args.no_extras:
         single = time_single_step_attention(ctx, device)  # before the long loop: at burst clocks, as a kernel timed alone
+        single_d64 = time_single_step_attention(ctx, device, head_dim=64)
     step = DeviceStep(ctx, w, seed=rank, device=device)
 
     sampler = ClockSampler(local_rank)
@@ -754,6 +759,15 @@ def main():
                     "frac": a_tf / peaks["bf16_tflops"], "ms": a_ms, "traffic": ncu_traffic("attention_ws_kernel", "single_step_bf16"),
                     "kernel": "attention_ws_kernel timed alone (20 launches back to back) on single_step_bf16: "
                               "16 heads, 4 chunks of 6240 tokens, all active, no clean region", "peak_kind": peak_kind + " burst"}
+            if single_d64 is not None:
+                a_ms, a_flops = single_d64
+                a_tf = a_flops / (a_ms * 1e-3) / 1e12
+                line["attention_single_step_bf16_d64"] = {
+                    "bound": "tensor", "achieved": a_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": a_tf / peaks["bf16_tflops"], "ms": a_ms, "traffic": None,
+                    "kernel": "attention_ws_kernel<64> timed alone (20 launches back to back): the single-step shape with "
+                              "32 heads of 64 instead of 16 of 128 (half the FLOPs per exponential)",
+                    "peak_kind": peak_kind + " burst"}
         if args.sweep:
             line["sweep"] = run_sweep(step, (0.05, 0.1, 0.2), 30, peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
         if args.streaming > 0:

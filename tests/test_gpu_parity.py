@@ -429,6 +429,37 @@ def test_attention_tensor_core_edge_cases(ctx, impl=2):
     assert torch.equal(Og.cpu(), O0)
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_attention_tensor_core_random_geometries(ctx, seed, impl=2):
+    # Seeded random layouts: head counts and grouping, head dimension, chunks of unequal (also zero) length, a logical
+    # key sequence cut into segments of random length laid out in shuffled physical order with gaps, visible lengths
+    # anywhere between nothing and everything, a random set of active chunks in random order.
+    rng = np.random.default_rng(1000 + seed)
+    d = int(rng.choice([64, 128]))
+    H_kv, group = int(rng.integers(1, 4)), int(rng.choice([1, 2]))
+    W = int(rng.integers(1, 7))
+    lens = rng.integers(0, 420, W)
+    lens[rng.integers(0, W)] += 1  # at least one row somewhere
+    q_off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    n_seg = int(rng.integers(1, 9))
+    seg_len = rng.integers(1, 300, n_seg)
+    slo = np.concatenate([[0], np.cumsum(seg_len)]).astype(np.int32)
+    phys, pos = np.zeros(n_seg, np.int32), int(rng.integers(0, 6))
+    for s_ in rng.permutation(n_seg):
+        phys[s_] = pos
+        pos += int(seg_len[s_]) + int(rng.integers(0, 40))
+    L_phys = pos + int(rng.integers(0, 5))
+    vis = rng.integers(0, slo[-1] + 1, W).astype(np.int32)
+    vis[rng.integers(0, W)] = slo[-1]
+    active = [int(c) for c in rng.permutation(W)[:int(rng.integers(1, W + 1))]]
+    Q = wl.normal((H_kv * group, int(q_off[-1]), d), 7000 + seed, 0.5, torch.bfloat16)
+    K = wl.normal((H_kv, L_phys, d), 7100 + seed, 0.5, torch.bfloat16)
+    V = wl.normal((H_kv, L_phys, d), 7200 + seed, 0.5, torch.bfloat16)
+    _poison_unreferenced_rows(K, V, int(vis.max()), slo, phys)
+    Og = _attention_custom(ctx, Q, K, V, q_off, vis, slo, phys, active, impl)
+    assert torch.isfinite(Og.float()).all()
+
+
 def _poison_unreferenced_rows(K, V, vis_max, slo, spo):
     """Overwrite every physical K/V row that no visible logical token maps to with NaN, +-inf and +-3e38."""
     L = K.shape[1]
@@ -791,6 +822,33 @@ def test_select_compact_tiny_and_ragged(ctx):
     wc = wl.Workload("c", "bf16", H=2, d=64, W=1, n_c=10, B=100, L_k=333, seed=6, sigma=0.5)
     _, Kc, Vc = wl.candidates(wc)
     _select_case(ctx, sb[:2, :333].copy(), 100, Kc, Vc)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_select_random_sizes_and_value_distributions(ctx, seed):
+    # Seeded random cases: lengths that do not divide by the cluster size or the vector width, budgets anywhere in
+    # [1, L], and score distributions that stress the radix passes: values quantised to a few levels (many ties, tie
+    # order decides), a range so narrow that all keys share their leading bits, a mix of signs, denormals and huge
+    # values, an already sorted head.
+    rng = np.random.default_rng(500 + seed)
+    H = int(rng.integers(1, 7))
+    L = int(rng.choice([1, 2, 31, 1023, 1025, 4097, 10007, 43681]))
+    kind = seed % 6
+    if kind == 0:
+        score = rng.integers(0, 4, size=(H, L)).astype(np.float32)
+    elif kind == 1:
+        score = (1.0 + rng.integers(0, 2000, size=(H, L)) * 2.0 ** -23).astype(np.float32)
+    elif kind == 2:
+        score = (rng.normal(size=(H, L)) * 10.0 ** rng.integers(-42, 38, size=(H, L)).astype(np.float64)).astype(np.float32)
+    elif kind == 3:
+        score = np.sort(rng.normal(size=(H, L)).astype(np.float32), axis=1)
+    elif kind == 4:
+        score = -np.abs(rng.normal(size=(H, L))).astype(np.float32)
+        score[:, ::7] = -0.0
+    else:
+        score = rng.random(size=(H, L)).astype(np.float32)
+    for B in sorted({1, max(1, L // 3), max(1, L - 1), L, int(rng.integers(1, L + 1))}):
+        assert _select_case(ctx, score, B) == 0
 
 
 def test_select_large_head_falls_back_to_global_keys(ctx):

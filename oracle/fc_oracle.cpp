@@ -313,12 +313,13 @@ extern "C" int fco_chunk_attention(
       s[j] = std::exp(s[j] - s_max);
       denom += s[j];
     }
-    for (int e = 0; e < d; ++e) {
-      double o = 0.0;
-      for (int32_t j = 0; j < n_vis; ++j)
-        o += s[j] * widen(V, dtype, (int64_t)h_kv * desc->v_hs + phys[j] * desc->v_rs + e);
-      out[e] = n_vis > 0 ? o / denom : 0.0;
+    // o = sum_j p_j v_j, one value row at a time (every component still adds its terms in the order j = 0, 1, ...)
+    std::vector<double> o(d, 0.0);
+    for (int32_t j = 0; j < n_vis; ++j) {
+      const int64_t v_row = (int64_t)h_kv * desc->v_hs + phys[j] * desc->v_rs;
+      for (int e = 0; e < d; ++e) o[e] += s[j] * widen(V, dtype, v_row + e);
     }
+    for (int e = 0; e < d; ++e) out[e] = n_vis > 0 ? o[e] / denom : 0.0;
     if (lse)
       lse[(int64_t)h * lse_hs + slots[idx]] =
           n_vis > 0 ? s_max + std::log(denom)

@@ -72,7 +72,7 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 // Four rows of a 2-D tensor (row indices r0..r3, starting at column c0) into four consecutive rows of a shared-memory
-// tile: the tile::gather4 form of the tiled load.  The tensor map's box is one row high.  No multicast.
+// tile: the tile::gather4 form of the tiled load.  The tensor map's box is one row high; the copy goes to this CTA only.
 __device__ __forceinline__ void tma_gather4_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int r0, int r1,
                                                int r2, int r3) {
   asm volatile(

@@ -527,14 +527,14 @@ def test_attention_bf16_many_items_per_cta(ctx, impl=2):
 
 # The launch configurations the benchmark times, at full size, on sampled query rows over the full key range:
 # boundary rows of every active chunk plus uniform draws from the active chunks (4096 on the single-step
-# configuration, 1024 on the others; the sparse sweep list and the second model family take 512).
+# configuration, 2048 on the others; the sparse sweep list and the second model family take 1024).
 FULL_SIZE_CASES = [
     ("single_step_bf16", [0, 1, 2, 3], 4096),
-    ("cached_step_bf16", [2, 5, 7], 1024),
-    ("streaming_bf16", [0], 1024),                 # one chunk over the 28080-token history
-    ("sweep_bf16", list(range(16)), 1024),         # every chunk of the window recomputed
-    ("sweep_bf16", [1, 4, 9, 15], 512),            # a sparse active list late in the sweep
-    ("skyreels_bf16", [0, 2, 3], 512),
+    ("cached_step_bf16", [2, 5, 7], 2048),
+    ("streaming_bf16", [0], 2048),                 # one chunk over the 28080-token history
+    ("sweep_bf16", list(range(16)), 2048),         # every chunk of the window recomputed
+    ("sweep_bf16", [1, 4, 9, 15], 1024),           # a sparse active list late in the sweep
+    ("skyreels_bf16", [0, 2, 3], 1024),
 ]
 
 
@@ -546,6 +546,14 @@ def test_attention_full_size_sampled_rows(ctx, name, active, n_uniform):
     assert len(rows) >= n_uniform * 0.9
     _attention_case(ctx, w, active, sample=rows, atol=1e-2, rel_l2=1e-2)
     torch.cuda.empty_cache()
+
+
+def test_attention_bf16_mid_size_every_element(ctx):
+    # every output element of a case with dozens of work items per head: 10 query tiles per chunk with a ragged
+    # last one, up to 52 key tiles per item, a clean region that ends inside a key tile
+    w = wl.Workload("mid", "bf16", H=4, d=128, W=4, n_c=1160, B=2000, L_k=3160, seed=18, sigma=0.5)
+    _attention_case(ctx, w, [0, 1, 2, 3], impl=2, atol=1e-2, rel_l2=1e-2)
+    _attention_case(ctx, w, [3, 1], impl=2, atol=1e-2, rel_l2=1e-2)
 
 
 def test_attention_bf16_matches_cuda_core_kernel(ctx):

@@ -724,6 +724,17 @@ def main():
                 "kernel": "score_mass_kernel x2 (row statistics, masses) + CUDA-core key statistics and "
                           "finalize (whole fc_kv_score call, outside the timed step); algorithmic FLOPs = "
                           "2 passes x 2 L_q L_k d H", "peak_kind": peak_kind + " burst"}
+            # the memory-bound calls again, timed back to back outside the step: what the copy rate they are compared
+            # with was measured as (a short kernel alone), without the clocks and cache state the 100 ms attention
+            # kernel leaves behind inside the step
+            for key, fn, nbytes in (("roofline_compact", step.select_compact, compact_bytes),
+                                    ("roofline_score", step.score_, step.L_k * w.d * es * w.H),
+                                    ("roofline_decide", step.decide, 2 * step.cur.numel() * es)):
+                a_ms = time_calls(fn, 20)
+                a_gbs = nbytes / (a_ms * 1e-3) / 1e9
+                line[key]["alone"] = {"ms": a_ms, "achieved": a_gbs, "frac": a_gbs / peaks["hbm_gbs"],
+                                      "frac_of_nominal": a_gbs / NOMINAL["hbm_gbs"],
+                                      "how": "the same call, 20 times back to back outside the timed step"}
             ca_ms, ca_bytes = time_cache_apply(step)
             ca_gbs = ca_bytes / (ca_ms * 1e-3) / 1e9
             line["roofline_cache_apply"] = {

@@ -38,23 +38,30 @@ constexpr int kDigitBits = 11, kBins = 1 << kDigitBits;  // at most three passes
 constexpr int kMaxCluster = 4;  // measured: a cluster of 8 is slower (25 us against 19 on 12 heads x 20400 keys)
 
 struct SelShared {
-  uint32_t hist[2][kBins];      // two copies (even / odd warps) to spread the atomics
-  uint32_t hist_cta[2][kBins];  // this CTA's histogram of the current digit, read by the other CTAs; passes alternate
-                                // between the two buffers, so one cluster barrier per pass is enough
+  uint32_t hist[2][kBins];  // this CTA's histogram of the current digit; two copies (even / odd warps) to spread the atomics
+  // Every CTA's histogram of the current digit, written into this CTA's shared memory by its owner (rank = second
+  // index) before the pass's cluster barrier and read locally after it.  Passes alternate between the two buffers, so
+  // one cluster barrier per pass is enough.
+  uint32_t hist_all[2][kMaxCluster][kBins];
   uint32_t red_min[kSelThreads / 32], red_max[kSelThreads / 32];
   uint32_t warp_gt[kSelThreads / 32], warp_eq[kSelThreads / 32], scan_w[kSelThreads / 32];
-  uint32_t cta_min, cta_max, cta_gt, cta_eq;  // read by the other CTAs
-  uint32_t prefix, remaining, nan;
+  uint32_t in_min[kMaxCluster], in_max[kMaxCluster];  // written by every CTA of the cluster: its smallest / largest key
+  uint32_t in_gt[kMaxCluster], in_eq[kMaxCluster];    // written by the CTAs that own lower indices: their kept counts
+  uint32_t prefix, remaining;
 };
 
+// Dynamic shared memory: SelShared, then (kSmemKeys) this CTA's keys.  No CTA reads another's shared memory: what the
+// others need is stored into THEIR shared memory before a cluster barrier, so the cost of the exchange is a store that
+// nobody waits for instead of a load across the cluster, and no CTA has to outlive its last barrier.
 template <bool kSmemKeys>
 __global__ void __launch_bounds__(kSelThreads)
 select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, int protect_from,
                    int32_t* __restrict__ kept_idx, int32_t* __restrict__ n_kept, uint32_t* __restrict__ status) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
-  extern __shared__ uint32_t smem_keys[];
-  __shared__ SelShared sh;
+  extern __shared__ __align__(16) uint8_t sel_smem[];
+  SelShared& sh = *reinterpret_cast<SelShared*>(sel_smem);
+  uint32_t* smem_keys = reinterpret_cast<uint32_t*>(sel_smem + sizeof(SelShared));
   const int cs = (int)cluster.num_blocks();
   const int rank = (int)cluster.block_rank(), h = blockIdx.x / cs, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
@@ -64,24 +71,25 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
 
   fc::pdl_launch_dependents();  // the gather's blocks may take their places; they wait for this grid to end
   fc::pdl_wait();               // the scores are complete and visible from here on
-  if (tid == 0) sh.nan = 0;
   if (tid == 0 && blockIdx.x == 0 && n_kept) *n_kept = B;
-  __syncthreads();
+  // the digit histograms start at zero; after that every pass clears what it has read
+  for (int b = tid; b < 2 * kBins; b += kSelThreads) (&sh.hist[0][0])[b] = 0;
   bool any_nan = false;
   // Keys, and their range.  The scores of a head sit in a narrow band, so their keys share the leading bits;
   // digits taken from the raw keys would send almost every key of the first passes to one histogram bin (and
   // one shared-memory atomic at a time).  The select therefore works on key - min(key), which keeps the order,
   // and starts at the highest bit in which the keys of this head differ.
   uint32_t kmin = 0xffffffffu, kmax = 0;
-  for (int j0 = tid; j0 < n; j0 += 4 * kSelThreads) {
-    float v[4];  // four loads in flight per thread
+  constexpr int kLoads = 12;  // loads in flight per thread: a quarter of a 44k-key head in one round
+  for (int j0 = tid; j0 < n; j0 += kLoads * kSelThreads) {
+    float v[kLoads];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kLoads; ++u) {
       const int j = j0 + u * kSelThreads;
       v[u] = j < n ? s[j] : 0.f;
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kLoads; ++u) {
       const int j = j0 + u * kSelThreads;
       if (j < n) {
         bool nn;
@@ -112,18 +120,18 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
       kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
       kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
     }
-    if (lane == 0) {
-      sh.cta_min = kmin;
-      sh.cta_max = kmax;
+    if (lane < cs) {  // lane q tells CTA q
+      SelShared* other = cluster.map_shared_rank(&sh, lane);
+      other->in_min[rank] = kmin;
+      other->in_max[rank] = kmax;
     }
   }
   cluster.sync();
   kmin = 0xffffffffu;
   kmax = 0;
   for (int q = 0; q < cs; ++q) {
-    const SelShared* other = cluster.map_shared_rank(&sh, q);
-    kmin = min(kmin, other->cta_min);
-    kmax = max(kmax, other->cta_max);
+    kmin = min(kmin, sh.in_min[q]);
+    kmax = max(kmax, sh.in_max[q]);
   }
   const uint32_t base = kmin;
   const int n_bits = kmax >= kmin ? 32 - __clz(kmax - kmin) : 0;  // 0 when all keys are equal
@@ -142,33 +150,27 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
   for (int hi = n_bits; hi > 0; ++pass) {
     const int lo = max(hi - kDigitBits, 0);
     const uint32_t digit_mask = (1u << (hi - lo)) - 1u;
-    for (int b = tid; b < 2 * kBins; b += kSelThreads) (&sh.hist[0][0])[b] = 0;
-    __syncthreads();
     for (int j = tid; j < n; j += kSelThreads) {
       const uint32_t k = key_at(j);
       const bool candidate = hi >= 32 || (k >> hi) == (prefix >> hi);
       if (candidate) atomicAdd(&sh.hist[warp & 1][(k >> lo) & digit_mask], 1u);
     }
     __syncthreads();
-    uint32_t* mine = sh.hist_cta[pass & 1];
-    for (int b = tid; b < kBins; b += kSelThreads) mine[b] = sh.hist[0][b] + sh.hist[1][b];
+    for (int b = tid; b < kBins; b += kSelThreads) {
+      const uint32_t v = sh.hist[0][b] + sh.hist[1][b];
+      sh.hist[0][b] = 0;  // for the next pass, whose atomics come after the barriers below
+      sh.hist[1][b] = 0;
+      for (int q = 0; q < cs; ++q) cluster.map_shared_rank(&sh, q)->hist_all[pass & 1][rank][b] = v;
+    }
     cluster.sync();
     {
       // digits from the largest downwards, two per thread; the digit of the B-th largest key is where the running
       // count first reaches `remaining`
       const int d0 = kBins - 1 - 2 * tid, d1 = d0 - 1;
-      uint32_t r0[kMaxCluster], r1[kMaxCluster];  // all remote loads in flight before the first add
-#pragma unroll
-      for (int q = 0; q < kMaxCluster; ++q) {
-        const SelShared* other = cluster.map_shared_rank(&sh, q < cs ? q : 0);
-        r0[q] = other->hist_cta[pass & 1][d0];
-        r1[q] = other->hist_cta[pass & 1][d1];
-      }
       uint32_t c0 = 0, c1 = 0;
-#pragma unroll
-      for (int q = 0; q < kMaxCluster; ++q) {
-        c0 += q < cs ? r0[q] : 0u;
-        c1 += q < cs ? r1[q] : 0u;
+      for (int q = 0; q < cs; ++q) {
+        c0 += sh.hist_all[pass & 1][q][d0];
+        c1 += sh.hist_all[pass & 1][q][d1];
       }
       const uint32_t tot = c0 + c1;
       uint32_t inc = tot;
@@ -202,61 +204,58 @@ select_topb_kernel(const float* __restrict__ score, int L_k, int B, int chunk, i
   const uint32_t T = prefix;           // key (relative to the minimum) of the B-th largest score
   const uint32_t need_eq = remaining;  // how many keys equal to T are kept (lowest indices)
 
-  // Ordered compaction: thread t owns the contiguous local range [t*per, (t+1)*per).
-  const int per = (n + kSelThreads - 1) / kSelThreads;
-  const int j0 = min(tid * per, n), j1 = min(j0 + per, n);
-  uint32_t n_gt = 0, n_eq = 0;
-  for (int j = j0; j < j1; ++j) {
-    const uint32_t k = key_at(j);
-    n_gt += k > T;
-    n_eq += k == T;
+  // Ordered compaction.  Warp w owns the contiguous local range [w * wper, (w + 1) * wper) and walks it 32 keys at a
+  // time: a ballot gives every kept key its rank among the 32, so the lanes of a warp write neighbouring entries of
+  // the output (one thread writing a run of entries of its own made every store instruction touch 32 sectors).
+  const int wper = (((n + 31) / 32 + 31) / 32) * 32;
+  const int w0 = min(warp * wper, n), w1 = min(w0 + wper, n);
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t n_gt = 0, n_eq = 0;  // of this warp's range (the same in every lane)
+  for (int j = w0 + lane; j - lane < w1; j += 32) {
+    const uint32_t k = j < w1 ? key_at(j) : 0u;
+    n_gt += __popc(__ballot_sync(0xffffffffu, j < w1 && k > T));
+    n_eq += __popc(__ballot_sync(0xffffffffu, j < w1 && k == T));
   }
-  // exclusive block scan of the packed pair (eq in the high half, gt in the low half)
-  uint32_t packed = (n_eq << 16) | n_gt;  // per-thread counts < 65536 (at most L_k/1024 items per thread)
-  uint32_t incl = packed;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += v;
-  }
-  // a warp's totals stay below 2^16 per half (L_k <= 2^20); block-level bases use full words
-  if (lane == 31) {
-    sh.warp_gt[warp] = incl & 0xffffu;
-    sh.warp_eq[warp] = incl >> 16;
+  if (lane == 0) {
+    sh.warp_gt[warp] = n_gt;
+    sh.warp_eq[warp] = n_eq;
   }
   __syncthreads();
-  uint32_t base_gt = lane < warp ? sh.warp_gt[lane] : 0u, base_eq = lane < warp ? sh.warp_eq[lane] : 0u;
+  // kept keys above T / equal to T in front of this warp: the warps before it, then the CTAs before this one
+  uint32_t gt_before = lane < warp ? sh.warp_gt[lane] : 0u, eq_before = lane < warp ? sh.warp_eq[lane] : 0u;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {  // totals of the warps in front of this one
-    base_gt += __shfl_xor_sync(0xffffffffu, base_gt, o);
-    base_eq += __shfl_xor_sync(0xffffffffu, base_eq, o);
+  for (int o = 16; o > 0; o >>= 1) {
+    gt_before += __shfl_xor_sync(0xffffffffu, gt_before, o);
+    eq_before += __shfl_xor_sync(0xffffffffu, eq_before, o);
   }
-  if (tid == kSelThreads - 1) {  // this CTA's totals, for the CTAs that own higher indices
-    sh.cta_gt = base_gt + (incl & 0xffffu);
-    sh.cta_eq = base_eq + (incl >> 16);
+  if (warp == kSelThreads / 32 - 1 && lane > rank && lane < cs) {
+    // This CTA's totals go into the shared memory of the CTAs that own higher indices (lane q tells CTA q).  Written
+    // before the barrier and read by their owner after it: no CTA touches another's shared memory after this barrier,
+    // so none has to wait for the others before it leaves.
+    SelShared* other = cluster.map_shared_rank(&sh, lane);
+    other->in_gt[rank] = gt_before + n_gt;
+    other->in_eq[rank] = eq_before + n_eq;
   }
   cluster.sync();
   for (int q = 0; q < rank; ++q) {
-    const SelShared* other = cluster.map_shared_rank(&sh, q);
-    base_gt += other->cta_gt;
-    base_eq += other->cta_eq;
+    gt_before += sh.in_gt[q];
+    eq_before += sh.in_eq[q];
   }
-  uint32_t gt_before = base_gt + (incl & 0xffffu) - n_gt;
-  uint32_t eq_before = base_eq + (incl >> 16) - n_eq;
-  for (int j = j0; j < j1; ++j) {
-    const uint32_t k = key_at(j);
-    if (k > T) {
-      const uint32_t pos = gt_before + min(eq_before, need_eq);
+  for (int j = w0 + lane; j - lane < w1; j += 32) {
+    const uint32_t k = j < w1 ? key_at(j) : 0u;
+    const bool gt = j < w1 && k > T, eq = j < w1 && k == T;
+    const uint32_t m_gt = __ballot_sync(0xffffffffu, gt), m_eq = __ballot_sync(0xffffffffu, eq);
+    const uint32_t gt_mine = gt_before + __popc(m_gt & lt), eq_mine = eq_before + __popc(m_eq & lt);
+    if (gt) {
+      const uint32_t pos = gt_mine + min(eq_mine, need_eq);
       if (fc::bounds_ok(pos < (uint32_t)B, status)) out[pos] = begin + j;
-      ++gt_before;
-    } else if (k == T) {
-      if (eq_before < need_eq && fc::bounds_ok(gt_before + eq_before < (uint32_t)B, status)) out[gt_before + eq_before] = begin + j;
-      ++eq_before;
+    } else if (eq && eq_mine < need_eq) {
+      if (fc::bounds_ok(gt_mine + eq_mine < (uint32_t)B, status)) out[gt_mine + eq_mine] = begin + j;
     }
+    gt_before += __popc(m_gt);
+    eq_before += __popc(m_eq);
   }
-  if (any_nan) sh.nan = 1;
-  cluster.sync();  // no CTA leaves while another may still read its shared memory
-  if (tid == 0 && sh.nan && status) atomicOr(status, FC_DEV_NAN_SCORE);
+  if (__any_sync(0xffffffffu, any_nan) && lane == 0 && status) atomicOr(status, FC_DEV_NAN_SCORE);
 }
 
 __global__ void select_identity_kernel(int32_t* __restrict__ kept_idx, int n_heads, int L_k,
@@ -367,10 +366,11 @@ int launch_select(fc_ctx* ctx, cudaStream_t st, const float* score, int n_heads,
   const int chunk = (L + cs - 1) / cs;
   const size_t key_bytes = (size_t)chunk * 4;
   const bool smem_keys = key_bytes + sizeof(SelShared) + 1024 <= (size_t)ctx->smem_optin;
+  const size_t smem_bytes = sizeof(SelShared) + (smem_keys ? key_bytes : 0);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)n_heads * cs);
   cfg.blockDim = dim3(kSelThreads);
-  cfg.dynamicSmemBytes = smem_keys ? key_bytes : 0;
+  cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -382,9 +382,10 @@ int launch_select(fc_ctx* ctx, cudaStream_t st, const float* score, int n_heads,
   cfg.attrs = attr;
   cfg.numAttrs = 2;
   if (smem_keys) {
-    FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+    FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
     FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<true>, score, L, B, chunk, protect_from, out_idx, n_kept, status));
   } else {
+    FC_CUDA_CHECK(cudaFuncSetAttribute(select_topb_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes));
     FC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, select_topb_kernel<false>, score, L, B, chunk, protect_from, out_idx, n_kept, status));
   }
   FC_LAUNCH_CHECK("select_topb_kernel");

@@ -861,9 +861,14 @@ def test_select_random_sizes_and_value_distributions(ctx, seed):
 
 def test_select_large_head_falls_back_to_global_keys(ctx):
     rng = np.random.default_rng(11)
-    score = rng.normal(size=(2, 70001)).astype(np.float32)  # 280 KB of keys: beyond shared memory
+    score = rng.normal(size=(2, 70001)).astype(np.float32)  # a cluster of four blocks per head, 70 KB of keys each
     score[:, ::3] = 0.5
     _select_case(ctx, score, 33333)
+    # 80 heads leave one block per head, and 60000 keys (240 KB) do not fit its shared memory: the keys are
+    # recomputed from the scores in global memory on every pass
+    score = rng.normal(size=(80, 60000)).astype(np.float32)
+    score[:, ::4] = -0.25
+    _select_case(ctx, score, 41234)
 
 
 def _select_units_case(ctx, score, B, unit, n_protect, K=None, V=None):

@@ -526,13 +526,13 @@ def test_attention_bf16_many_items_per_cta(ctx, impl=2):
 
 
 # The launch configurations the benchmark times, at full size, on sampled query rows over the full key range:
-# boundary rows of every active chunk plus uniform draws from the active chunks (4096 on the single-step
-# configuration, 2048 on the others; the sparse sweep list and the second model family take 1024).
+# boundary rows of every active chunk plus uniform draws from the active chunks (4096 distinct rows on each of the
+# four full-size configurations; the extra cases, a sparse sweep list and the second model family, take 1024).
 FULL_SIZE_CASES = [
     ("single_step_bf16", [0, 1, 2, 3], 4096),
-    ("cached_step_bf16", [2, 5, 7], 2048),
-    ("streaming_bf16", [0], 2048),                 # one chunk over the 28080-token history
-    ("sweep_bf16", list(range(16)), 2048),         # every chunk of the window recomputed
+    ("cached_step_bf16", [2, 5, 7], 4096),
+    ("streaming_bf16", [0], 4096),                 # one chunk over the 28080-token history
+    ("sweep_bf16", list(range(16)), 4096),         # every chunk of the window recomputed
     ("sweep_bf16", [1, 4, 9, 15], 1024),           # a sparse active list late in the sweep
     ("skyreels_bf16", [0, 2, 3], 1024),
 ]

@@ -363,8 +363,11 @@ def time_device(step, steps, warmup, barrier):
     torch.cuda.synchronize()
     barrier()
     total_ms = t0.elapsed_time(t1)
-    stage_ms = {name: statistics.mean(ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(steps))
-                for i, name in enumerate(DeviceStep.STAGES)}
+    per_stage = {name: [ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(steps)]
+                 for i, name in enumerate(DeviceStep.STAGES)}
+    stage_ms = {name: statistics.mean(v) for name, v in per_stage.items()}
+    stage_ms["median"] = {name: statistics.median(v) for name, v in per_stage.items()}
+    stage_ms["best"] = {name: min(v) for name, v in per_stage.items()}
     return total_ms, stage_ms
 
 

@@ -129,9 +129,24 @@ decide_finalize_kernel(DecideGeom g, const double2* __restrict__ partial,
     const int c = c0 + warp / wpc, sub = warp % wpc;
     double num = 0.0, den = 0.0;
     if (c < g.n_chunks) {
-      for (int s = g.slab_off[c] + sub * 32 + lane; s < g.slab_off[c + 1]; s += wpc * 32) {
-        num += partial[s].x;
-        den += partial[s].y;
+      // eight loads in flight at a time (one after the other, every iteration waited for its own load: 37 round trips
+      // on 16 chunks of 2340 slabs); the additions keep their order
+      constexpr int kBatch = 8;
+      const int end = g.slab_off[c + 1], stride = wpc * 32;
+      for (int s0 = g.slab_off[c] + sub * 32 + lane; s0 < end; s0 += kBatch * stride) {
+        double2 v[kBatch];
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+          const int s = s0 + k * stride;
+          v[k] = s < end ? partial[s] : make_double2(0.0, 0.0);
+        }
+#pragma unroll
+        for (int k = 0; k < kBatch; ++k) {
+          if (s0 + k * stride < end) {
+            num += v[k].x;
+            den += v[k].y;
+          }
+        }
       }
     }
 #pragma unroll

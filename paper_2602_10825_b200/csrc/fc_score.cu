@@ -240,11 +240,20 @@ score_finalize_kernel(ScoreGeom g, const float* __restrict__ imp_in, const float
   const int hk = blockIdx.y, tid = threadIdx.x;
   fc::pdl_wait();  // launched under the tail of the kernel that writes imp, a and the softmax statistics
   float m = -INFINITY, l = 0.f;
-  for (int t = tid; t < g.n_partials; t += kFinThreads) {
-    const float2 p = a_partial[hk * g.n_partials + t];
-    const float mn = fmaxf(m, p.x);
-    l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * expf(p.x - mn));
-    m = mn;
+  for (int t0 = tid; t0 < g.n_partials; t0 += 8 * kFinThreads) {  // eight loads in flight, merged in the same order
+    float2 p[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int t = t0 + k * kFinThreads;
+      p[k] = t < g.n_partials ? a_partial[hk * g.n_partials + t] : make_float2(-INFINITY, 0.f);
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if (t0 + k * kFinThreads >= g.n_partials) break;
+      const float mn = fmaxf(m, p[k].x);
+      l = (m == -INFINITY ? 0.f : l * expf(m - mn)) + (p[k].x == -INFINITY ? 0.f : p[k].y * expf(p[k].x - mn));
+      m = mn;
+    }
   }
   reduce_ml<kFinThreads>(m, l, sm_m, sm_l);
   if (tid == 0) {

@@ -107,25 +107,8 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
     tma_prefetch_desc(&tmap_q);
     tma_prefetch_desc(&tmap_k);
   }
-  // Both passes let their successor (pass 2, the finalize kernel) be scheduled under their tail; pass 2 is such a
-  // successor itself and waits here, its barriers already initialised, for pass 1's results to be complete.
+  // Both passes let their successor (pass 2, the finalize kernel) be scheduled under their tail.
   fc::pdl_launch_dependents();
-  if (PASS == 2) fc::pdl_wait();
-  if (PASS == 2 && tid < kNQ) {
-    // log-sum-exp of query `tid` over the whole head: pass 1's per-slice (max, sum) pairs, merged in slice order
-    float lse = INFINITY;  // padding queries: exp2(anything - inf) = 0
-    if (tid < g.L_q) {
-      float m = -INFINITY, l = 0.f;
-      for (int s = 0; s < g.n_slices; ++s) {
-        const float2 p = g.ml_part[((int64_t)hk * g.n_slices + s) * kNQ + tid];
-        const float mn = fmaxf(m, p.x);
-        l = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p.x == -INFINITY ? 0.f : p.y * exp2f(p.x - mn));
-        m = mn;
-      }
-      lse = m + log2f(l);
-    }
-    sh->lse_s[tid] = -lse;
-  }
   if (warp == 0) {
     tmem_alloc(smem_u32(&sh->tmem_base), 2 * kCols);
     tmem_relinquish();
@@ -133,6 +116,33 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  // Pass 2 is such a successor itself.  Its copy warp touches nothing that pass 1 writes (keys and queries are the
+  // call's inputs), so it starts filling the key ring at once, under pass 1's tail; every other warp waits here for
+  // pass 1's results to be complete and visible.
+  if (PASS == 2 && warp != kCopyWarp<PASS>) fc::pdl_wait();
+  if (PASS == 2 && tid < kNQ) {
+    // log-sum-exp of query `tid` over the whole head: pass 1's per-slice (max, sum) pairs, merged in slice order
+    // (loaded eight at a time: one dependent round trip per slice would cost microseconds before the first tile)
+    float lse = INFINITY;  // padding queries: exp2(anything - inf) = 0
+    if (tid < g.L_q) {
+      float m = -INFINITY, l = 0.f;
+      for (int s0 = 0; s0 < g.n_slices; s0 += 8) {
+        float2 p[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          p[k] = s0 + k < g.n_slices ? g.ml_part[((int64_t)hk * g.n_slices + s0 + k) * kNQ + tid] : make_float2(-INFINITY, 0.f);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          if (s0 + k >= g.n_slices) break;
+          const float mn = fmaxf(m, p[k].x);
+          l = (m == -INFINITY ? 0.f : l * exp2f(m - mn)) + (p[k].x == -INFINITY ? 0.f : p[k].y * exp2f(p[k].x - mn));
+          m = mn;
+        }
+      }
+      lse = m + log2f(l);
+    }
+    sh->lse_s[tid] = -lse;
+  }
   const uint32_t tmem = sh->tmem_base;
 
   if (warp == kCopyWarp<PASS>) {
@@ -251,10 +261,19 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       // The mean key joins the queries as rows kNQ-2 (bf16 high part) and kNQ-1 (low part) of the Q tile, which
       // the copy zero-filled: generic-proxy writes, made visible to the tensor cores by the proxy fence.
       const int wg = warp >> 2, row = tid & 127;
+      asm volatile("bar.sync 5, 256;" ::: "memory");  // lse_s, written by warps 0 and 1 above, is read by all eight
       if (wg == 0) mbar_wait_bounded(smem_u32(&sh->q_full), 0, abort);
       if (tid < D) {
         float mk = 0.f;  // mean normalised key: pass 1's per-slice column sums, added in slice order
-        for (int s = 0; s < g.n_slices; ++s) mk += g.colsum_part[((int64_t)hk * g.n_slices + s) * D + tid];
+        for (int s0 = 0; s0 < g.n_slices; s0 += 8) {
+          float v[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            v[k] = s0 + k < g.n_slices ? g.colsum_part[((int64_t)hk * g.n_slices + s0 + k) * D + tid] : 0.f;
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            if (s0 + k < g.n_slices) mk += v[k];
+        }
         mk /= (float)g.L_k;
         const __nv_bfloat16 hi = __float2bfloat16_rn(mk), lo = __float2bfloat16_rn(mk - __bfloat162float(hi));
         const int c = tid >> 3, x = c >> 3, cc = c & 7, e = tid & 7;

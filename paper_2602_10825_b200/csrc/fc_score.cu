@@ -162,13 +162,194 @@ score_row_lse_kernel(const float* __restrict__ S, int L_k, float* __restrict__ l
   if (threadIdx.x == 0) lse[row] = m + logf(l);
 }
 
-__global__ void score_mean_key_kernel(const float* __restrict__ mk_partial, int n_tiles, int d, int L_k,
-                                      float* __restrict__ mean_key) {
-  const int hk = blockIdx.x, e = threadIdx.x;
-  if (e >= d) return;
+// Mean normalised key of a head from the per-tile sums.  One block per head, kMkGroups x 128 threads: group r adds
+// the tiles r, r + kMkGroups, ... (eight loads in flight; one thread per component walking all tiles waited for one
+// load after the other, 342 of them on 43680 keys), the groups are added in group order.  Fixed order throughout.
+constexpr int kMkGroups = 8;
+__global__ void __launch_bounds__(kMkGroups * 128)
+score_mean_key_kernel(const float* __restrict__ mk_partial, int n_tiles, int d, int L_k,
+                      float* __restrict__ mean_key) {
+  __shared__ float part[kMkGroups][128];
+  const int hk = blockIdx.x, e = threadIdx.x & 127, r = threadIdx.x >> 7;
   float acc = 0.f;
-  for (int t = 0; t < n_tiles; ++t) acc += mk_partial[((int64_t)hk * n_tiles + t) * d + e];
-  mean_key[hk * d + e] = acc / (float)L_k;
+  if (e < d) {
+    const float* src = mk_partial + (int64_t)hk * n_tiles * d + e;
+    for (int t0 = r; t0 < n_tiles; t0 += 8 * kMkGroups) {
+      float v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int t = t0 + k * kMkGroups;
+        v[k] = t < n_tiles ? src[(int64_t)t * d] : 0.f;
+      }
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (t0 + k * kMkGroups < n_tiles) acc += v[k];
+    }
+  }
+  part[r][e] = acc;
+  __syncthreads();
+  if (r == 0 && e < d) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < kMkGroups; ++q) t += part[q][e];
+    mean_key[hk * d + e] = t / (float)L_k;
+  }
+}
+
+// ---- frame-level pipeline: the two sweeps over the keys around the tensor-core launches (bf16) ----------------
+// A warp reads whole rows with one instruction: a key row is D / 8 chunks of 16 bytes, one per lane, so a warp
+// instruction covers 32 / (D / 8) consecutive rows (512 contiguous bytes).  What a row needs as a whole (its squared
+// norm, its product with the mean key) is a sum over the lanes that hold it: log2(D / 8) shuffle steps.
+template <int D>
+struct RowLanes {
+  static constexpr int kLanes = D / 8;        // lanes per row
+  static constexpr int kRows = 32 / kLanes;   // rows per warp instruction
+};
+
+__device__ __forceinline__ void unpack8(const uint4& w, float (&x)[8]) {
+  const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    x[2 * i] = fc::bf16_lo(ww[i]);
+    x[2 * i + 1] = fc::bf16_hi(ww[i]);
+  }
+}
+
+// Sums of the l2-normalised keys of one tile: mk_partial[head, tile, D] (what score_pass1_kernel leaves, without
+// its logits).  128 threads, warp w takes rows 32 w .. 32 w + 31 of the tile.  Three steps: the squared norm of every
+// row (lanes of a row added by shuffles) into shared memory; one reciprocal norm per thread (the square root and
+// the division once per row, all lanes busy); the rows, still in registers, scaled and added up per column.
+template <int D>
+__global__ void __launch_bounds__(kTile)
+frame_key_sums_kernel(const __nv_bfloat16* __restrict__ K, ScoreGeom g, float* __restrict__ mk_partial) {
+  constexpr int kLanes = RowLanes<D>::kLanes, kRows = RowLanes<D>::kRows, kIters = 32 / kRows;
+  __shared__ float part[kTile / 32][D];
+  __shared__ float n2_s[kTile];  // squared norms, then reciprocal norms
+  const int hk = blockIdx.y, tile = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane % kLanes, rsel = lane / kLanes;
+  const __nv_bfloat16* base = K + (int64_t)hk * g.k_hs + sub * 8;
+  uint4 w[kIters];
+#pragma unroll
+  for (int it = 0; it < kIters; ++it) {  // all loads of the warp's 32 rows first
+    const int row = tile * kTile + warp * 32 + it * kRows + rsel;
+    w[it] = row < g.L_k ? __ldg(reinterpret_cast<const uint4*>(base + (int64_t)row * g.k_rs)) : make_uint4(0u, 0u, 0u, 0u);
+  }
+#pragma unroll
+  for (int it = 0; it < kIters; ++it) {
+    float x[8];
+    unpack8(w[it], x);
+    float n2 = 0.f;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) n2 = fmaf(x[e], x[e], n2);
+#pragma unroll
+    for (int o = kLanes / 2; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+    if (sub == 0) n2_s[warp * 32 + it * kRows + rsel] = n2;
+  }
+  __syncthreads();
+  n2_s[threadIdx.x] = 1.f / fmaxf(sqrtf(n2_s[threadIdx.x]), 1e-12f);  // rows past the end are zeros: 0 * 1e12 = 0
+  __syncthreads();
+  float acc[8];
+#pragma unroll
+  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll
+  for (int it = 0; it < kIters; ++it) {
+    float x[8];
+    unpack8(w[it], x);
+    const float inv = n2_s[warp * 32 + it * kRows + rsel];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = fmaf(x[e], inv, acc[e]);
+  }
+  // the lanes that hold the same chunk of different rows, then the warps, in a fixed order
+#pragma unroll
+  for (int o = kLanes; o < 32; o <<= 1)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+  if (rsel == 0)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) part[warp][sub * 8 + e] = acc[e];
+  __syncthreads();
+  if (threadIdx.x < D) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < kTile / 32; ++q) t += part[q][threadIdx.x];
+    mk_partial[((int64_t)hk * g.n_tiles + tile) * D + threadIdx.x] = t;
+  }
+}
+
+// After the mass launch: importance = mass / n_q (with the accumulation over steps), redundancy argument
+// a_j = meankey . khat_j - |khat_j|^2 / L_k and its per-tile softmax statistics (what score_pass2_kernel does with
+// one key per thread and uncoalesced row loads).  Two steps: the warps sweep the rows (squared norm and product with
+// the mean key of every row, by shuffles, into shared memory); then one key per thread, so that the square root,
+// the division and every access to the per-key arrays are done by all threads at once.
+template <int D>
+__global__ void __launch_bounds__(kTile)
+frame_finish_kernel(const __nv_bfloat16* __restrict__ K, ScoreGeom g, const float* __restrict__ mean_key,
+                    const float* __restrict__ mass_in, float* __restrict__ imp_accum, int accum_phase, int n_steps,
+                    float* __restrict__ imp_out, float* __restrict__ a_out, float2* __restrict__ a_partial) {
+  constexpr int kLanes = RowLanes<D>::kLanes, kRows = RowLanes<D>::kRows, kIters = 32 / kRows;
+  __shared__ float sm_m[kTile / 32], sm_l[kTile / 32];
+  __shared__ float n2_s[kTile], dot_s[kTile];
+  const int hk = blockIdx.y, tile = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int j = tile * kTile + tid;
+  const bool valid = j < g.L_k;
+  const int64_t o = (int64_t)hk * g.L_k + j;
+  if (valid) {
+    const float ms = mass_in[o] / (float)g.n_q;
+    if (accum_phase == 1) {
+      imp_accum[o] += ms;
+    } else if (accum_phase == 2) {
+      const float t = imp_accum[o] + ms;
+      imp_accum[o] = t;
+      imp_out[o] = t / (float)n_steps;
+    } else {
+      imp_out[o] = ms;
+    }
+  }
+  if (accum_phase == 1) return;
+  {
+    const int sub = lane % kLanes, rsel = lane / kLanes;
+    const __nv_bfloat16* base = K + (int64_t)hk * g.k_hs + sub * 8;
+    float mk[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mk[e] = mean_key[hk * D + sub * 8 + e];
+    uint4 w[kIters];
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+      const int row = tile * kTile + warp * 32 + it * kRows + rsel;
+      w[it] = row < g.L_k ? __ldg(reinterpret_cast<const uint4*>(base + (int64_t)row * g.k_rs)) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int it = 0; it < kIters; ++it) {
+      float x[8];
+      unpack8(w[it], x);
+      float n2 = 0.f, dot = 0.f;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        n2 = fmaf(x[e], x[e], n2);
+        dot = fmaf(mk[e], x[e], dot);
+      }
+#pragma unroll
+      for (int o2 = kLanes / 2; o2 > 0; o2 >>= 1) {
+        n2 += __shfl_xor_sync(0xffffffffu, n2, o2);
+        dot += __shfl_xor_sync(0xffffffffu, dot, o2);
+      }
+      if (sub == 0) {
+        n2_s[warp * 32 + it * kRows + rsel] = n2;
+        dot_s[warp * 32 + it * kRows + rsel] = dot;
+      }
+    }
+  }
+  __syncthreads();
+  float a = -INFINITY;
+  if (valid) {
+    const float n2 = n2_s[tid];
+    const float inv = 1.f / fmaxf(sqrtf(n2), 1e-12f);
+    a = dot_s[tid] * inv - (n2 * inv * inv) / (float)g.L_k;
+    a_out[o] = a;
+  }
+  float m = a, l = valid ? 1.f : 0.f;
+  reduce_ml<kTile>(m, l, sm_m, sm_l);
+  if (tid == 0) a_partial[hk * g.n_tiles + tile] = make_float2(m, l);
 }
 
 template <typename T, int D>
@@ -356,7 +537,7 @@ int run(cudaStream_t st, const ScoreGeom& g, const ScoreWs& w, const void* Q, co
   FC_LAUNCH_CHECK("score_pass1_kernel");
   score_row_lse_kernel<<<dim3(g.n_q, g.H_kv), 256, 0, st>>>(w.S, g.L_k, w.lse);
   FC_LAUNCH_CHECK("score_row_lse_kernel");
-  score_mean_key_kernel<<<g.H_kv, 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
+  score_mean_key_kernel<<<g.H_kv, kMkGroups * 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
   FC_LAUNCH_CHECK("score_mean_key_kernel");
   score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, w.S, w.lse, w.mean_key, nullptr, imp_accum, phase,
                                                    n_steps, imp_buf, w.a, w.a_partial);
@@ -370,23 +551,19 @@ int run_frame(fc_ctx* ctx, cudaStream_t st, const ScoreGeom& g, const ScoreWs& w
               float* imp_accum, int phase, int n_steps, float* imp_buf, uint32_t* status) {
   using T = __nv_bfloat16;
   dim3 grid(g.n_tiles, g.H_kv);
-  // 1. sums of normalised keys per tile (no queries: the logit loop of the kernel is empty)
-  ScoreGeom g0 = g;
-  g0.n_q = 0;
-  const size_t smem1 = (size_t)kTile * (D + 1) * 4;
-  FC_CUDA_CHECK(cudaFuncSetAttribute(score_pass1_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1));
-  score_pass1_kernel<T, D><<<grid, kTile, smem1, st>>>((const T*)Q, (const T*)K, g0, nullptr, w.mk_partial);
-  FC_LAUNCH_CHECK("score_pass1_kernel");
-  score_mean_key_kernel<<<g.H_kv, 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
+  // 1. sums of normalised keys per tile, then the head's mean key
+  frame_key_sums_kernel<D><<<grid, kTile, 0, st>>>((const T*)K, g, w.mk_partial);
+  FC_LAUNCH_CHECK("frame_key_sums_kernel");
+  score_mean_key_kernel<<<g.H_kv, kMkGroups * 128, 0, st>>>(w.mk_partial, g.n_tiles, D, g.L_k, w.mean_key);
   FC_LAUNCH_CHECK("score_mean_key_kernel");
   // 2., 3. log-sum-exp of every query over the candidates, then the attention mass of every key
   int rc = fc::score_frame_mass(ctx, st, g.H_kv, g.d, g.L_q, g.L_k, g.scale * 1.4426950408889634f, Q, g.q_hs, g.q_rs, K,
                                 g.k_hs, g.k_rs, w.fr_ml, w.lse, w.fr_mass, status);
   if (rc != FC_OK) return rc;
   // 4. mean over the queries, accumulation over steps, redundancy logits
-  score_pass2_kernel<T, D><<<grid, kTile, 0, st>>>((const T*)K, g, nullptr, nullptr, w.mean_key, w.fr_mass, imp_accum,
-                                                   phase, n_steps, imp_buf, w.a, w.a_partial);
-  FC_LAUNCH_CHECK("score_pass2_kernel");
+  frame_finish_kernel<D><<<grid, kTile, 0, st>>>((const T*)K, g, w.mean_key, w.fr_mass, imp_accum, phase, n_steps, imp_buf,
+                                                 w.a, w.a_partial);
+  FC_LAUNCH_CHECK("frame_finish_kernel");
   return FC_OK;
 }
 

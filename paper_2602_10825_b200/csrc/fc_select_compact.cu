@@ -14,6 +14,7 @@
 // dependent of the selection: its blocks take their places on the SMs while the selection still runs and start
 // copying the moment it has ended.
 #include <algorithm>
+#include <cstdint>
 
 #include <cooperative_groups.h>
 
@@ -281,23 +282,27 @@ constexpr int kUnroll = 4;
 __global__ void __launch_bounds__(kCopyThreads)
 gather_rows_kernel(const uint8_t* __restrict__ K_src, const uint8_t* __restrict__ V_src,
                    uint8_t* __restrict__ K_dst, uint8_t* __restrict__ V_dst,
-                   const int32_t* __restrict__ kept_idx, int n_keep, int L_k, int pieces_per_row,
+                   const int32_t* __restrict__ kept_idx, int n_keep, int L_k, int pieces_per_row, int ppr_shift,
                    int64_t src_hs_b, int64_t src_rs_b, int64_t dst_hs_b, int64_t dst_rs_b,
                    uint32_t* __restrict__ status) {
   const int h = blockIdx.y;
   fc::pdl_wait();  // the kept indices are complete and visible from here on
-  const int64_t n_pieces = (int64_t)n_keep * pieces_per_row;
-  const int64_t p0 = (int64_t)blockIdx.x * (kCopyThreads * kUnroll) + threadIdx.x;
+  // piece numbers fit 32 bits (the launcher checks), and a row is a power of two of pieces for every power-of-two head
+  // dimension (ppr_shift >= 0): a shift and a mask instead of divisions, which cost more than the copy's own
+  // instructions and show once the clocks are low
+  const uint32_t n_pieces = (uint32_t)n_keep * (uint32_t)pieces_per_row;
+  const uint32_t p0 = blockIdx.x * (uint32_t)(kCopyThreads * kUnroll) + threadIdx.x;
   const int32_t* idx = kept_idx + (size_t)h * n_keep;
   uint4 kv[kUnroll], vv[kUnroll];
   int64_t dst_off[kUnroll];
   bool ok[kUnroll];
 #pragma unroll
   for (int u = 0; u < kUnroll; ++u) {
-    const int64_t p = p0 + (int64_t)u * kCopyThreads;
+    const uint32_t p = p0 + (uint32_t)u * kCopyThreads;
     ok[u] = p < n_pieces;
     if (ok[u]) {
-      const int r = (int)(p / pieces_per_row), c = (int)(p % pieces_per_row);
+      const int r = (int)(ppr_shift >= 0 ? p >> ppr_shift : p / (uint32_t)pieces_per_row);
+      const int c = (int)(p - (uint32_t)r * (uint32_t)pieces_per_row);
       const int32_t src_row = idx[r];
       if (src_row < 0 || src_row >= L_k) {  // never produced by the selection kernel
         ok[u] = false;
@@ -421,9 +426,14 @@ int launch_gather(cudaStream_t st, const CopyArgs& c, const int32_t* kept_idx, i
   const int es = fc::elem_size(c.dtype);
   const int ppr = c.d * es / 16;
   const int64_t n_pieces = (int64_t)n_keep * ppr;
+  if (n_pieces + kCopyThreads * kUnroll > (int64_t)UINT32_MAX) return FC_ERR_UNSUPPORTED;  // 64 GB of rows per head and tensor
+  int ppr_shift = -1;
+  for (int sft = 0; sft < 16; ++sft)
+    if ((1 << sft) == ppr) ppr_shift = sft;
   dim3 grid((unsigned)((n_pieces + kCopyThreads * kUnroll - 1) / (kCopyThreads * kUnroll)), n_heads);
   FC_CUDA_CHECK(fc::launch_pdl(gather_rows_kernel, grid, dim3(kCopyThreads), 0, st, (const uint8_t*)c.K_src,
                                (const uint8_t*)c.V_src, (uint8_t*)c.K_dst, (uint8_t*)c.V_dst, kept_idx, n_keep, L_k, ppr,
+                               ppr_shift,
                                c.strides->src_hs * es, c.strides->src_rs * es, c.strides->dst_hs * es,
                                c.strides->dst_rs * es, status));
   FC_LAUNCH_CHECK("gather_rows_kernel");

@@ -7,7 +7,8 @@
 // each) finds the key T of the B-th largest score and how many keys exceed it; one ordered
 // compaction then keeps every key above T plus the lowest-index keys equal to T, so the kept
 // set is exactly the first B elements of the total order (score descending, index ascending),
-// written in ascending index order.  Integer work only: bit-exact.
+// written in ascending index order (by warps, 32 neighbouring entries at a time, positions from ballots).  Integer
+// work only: bit-exact.
 //
 // Compaction: a separate streaming kernel moves whole rows with 16-byte accesses, several
 // independent loads in flight per thread; rows that were dropped are never read.  It is launched as a programmatic
@@ -34,9 +35,10 @@ __device__ __forceinline__ uint32_t score_key(float s, bool& is_nan) {
 
 // One cluster of CTAs per head (1, 2 or 4 of them: as many as keep the whole grid within one wave); CTA r of the
 // cluster owns the contiguous index range [r * chunk, (r + 1) * chunk) of the head.  The CTAs exchange their partial
-// results (minimum / maximum, digit histograms, counts of kept keys) by reading each other's shared memory.
+// results (minimum / maximum, digit histograms, counts of kept keys) by storing them into each other's shared
+// memory before a cluster barrier.
 constexpr int kDigitBits = 11, kBins = 1 << kDigitBits;  // at most three passes over 32 bits
-constexpr int kMaxCluster = 4;  // measured: a cluster of 8 is slower (25 us against 19 on 12 heads x 20400 keys)
+constexpr int kMaxCluster = 4;  // measured: a cluster of 8 is slower (16.6 us against 13.2 on 12 heads x 20400 keys)
 
 struct SelShared {
   uint32_t hist[2][kBins];  // this CTA's histogram of the current digit; two copies (even / odd warps) to spread the atomics

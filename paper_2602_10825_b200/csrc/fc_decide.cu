@@ -6,8 +6,9 @@
 // tail and waits there).  (1) A streaming segmented reduction: the chunks are cut into slabs of 16 KiB
 // per tensor, one block per slab; every thread sums |cur-prev| and |prev| of 4 interleaved
 // 16-byte vectors in fp32, the block combines them in fp64 in a fixed tree and writes one
-// (num, den) pair per slab.  (2) One block: a warp per chunk adds that chunk's slab pairs in a
-// fixed order in fp64, forms r, applies the rule in fp32 and compacts the active ids.
+// (num, den) pair per slab.  (2) One block: its 32 warps are shared out over the chunks; they add a chunk's slab
+// pairs in a fixed order in fp64 (eight loads in flight per thread), form r, apply the rule in fp32 and compact the
+// active ids.
 // No atomics: results are bit-reproducible from run to run.
 #include <atomic>
 

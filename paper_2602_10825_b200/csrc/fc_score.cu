@@ -6,10 +6,10 @@
 // kernel below; everything else (fp32, more queries, grouped query heads whose rows are not contiguous) takes the
 // CUDA-core pipeline (below).  Grouped query heads stored head after head are folded into one head of group * L_q
 // queries first, so they take whichever pipeline that number of queries takes.  bf16 inputs with more than 128 observation queries per key head (a latent frame
-// or a whole chunk of them) take the frame-level pipeline: key norms and mean key by the CUDA-core pass-1 kernel
-// without queries, every query's log-sum-exp over the candidates and then the attention mass of every key by the
-// tensor-core kernel of fc_score_frame.cu (two launches), then the CUDA-core pass-2 kernel fed with that mass, and
-// the finalize kernel.
+// or a whole chunk of them) take the frame-level pipeline: sums of normalised keys and the mean key by
+// frame_key_sums_kernel and score_mean_key_kernel (below), every query's log-sum-exp over the candidates and then the
+// attention mass of every key by the tensor-core kernel of fc_score_frame.cu (two launches), then frame_finish_kernel
+// (below: importance from that mass, redundancy argument) and the finalize kernel.
 // The CUDA-core pipeline, five launches per call:
 //   pass1     one thread per key: raw logits of all observation queries against its key,
 //             written to the workspace; normalised key summed per 128-key tile (mean key)

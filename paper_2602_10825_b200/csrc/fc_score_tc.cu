@@ -22,8 +22,8 @@
 // memory and two read the key tile from shared memory (norms, column sums), each pair taking alternate tiles; one
 // warp streams key tiles through a 4-stage TMA ring and issues the MMAs into a 2-deep tensor-memory ring (one
 // accumulator per logit warpgroup).  Pass 2 (288 threads): no key-vector work, two logit warpgroups on alternate
-// tiles.  Keys are read from HBM once: the second pass finds them in L2 for the cache sizes of the paper (a head is
-// a few MB).
+// tiles.  The second pass walks heads, slices and tiles in the reverse of the first pass's order, so it starts on
+// what the first pass left in L2 (all of it while the candidates of all heads fit there: a head is a few MB).
 // Sums are fixed-order: results are bit-reproducible from run to run.  Every mbarrier wait is bounded.
 #include <cmath>
 

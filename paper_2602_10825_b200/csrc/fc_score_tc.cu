@@ -352,26 +352,31 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
       // column sums of the normalised keys: this thread owns 16-byte chunk `c` of the rows r = rg (mod kGroups)
       constexpr int kGroups = 128 / kChunks;  // 8 for d = 128, 16 for d = 64
       const int c = u % kChunks, rg = u / kChunks;
-      float acc[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+      uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};  // columns (2e, 2e + 1) of this thread's chunk
       for (int i = vg; i < n; i += 2) {
         const int st = i % kRing;
         mbar_wait_bounded(smem_u32(&sh->k_full[st]), (i / kRing) & 1, abort);
         const uint8_t* tile = k_tiles + st * kTileBytes;
-        float n4[4] = {0.f, 0.f, 0.f, 0.f};
+        uint64_t n4[4] = {0ull, 0ull, 0ull, 0ull};  // two-wide fp32: (low element, high element) of each 32-bit word
 #pragma unroll
         for (int cc = 0; cc < kChunks; ++cc) {
           const uint4 w = lds_key_chunk<D>(tile, u, cc);
           const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float lo = fc::bf16_lo(ww[e]), hi = fc::bf16_hi(ww[e]);
-            n4[e] = fmaf(lo, lo, n4[e]);
-            n4[e] = fmaf(hi, hi, n4[e]);
+            const uint64_t p2 = pack2(fc::bf16_lo(ww[e]), fc::bf16_hi(ww[e]));
+            n4[e] = fma2(p2, p2, n4[e]);
           }
         }
-        const float n2 = (n4[0] + n4[1]) + (n4[2] + n4[3]);
+        float n2;
+        {
+          float a0, a1, b0, b1, c0, c1, d0, d1;
+          unpack2(n4[0], a0, a1);
+          unpack2(n4[1], b0, b1);
+          unpack2(n4[2], c0, c1);
+          unpack2(n4[3], d0, d1);
+          n2 = ((a0 + a1) + (b0 + b1)) + ((c0 + c1) + (d0 + d1));
+        }
         const int j = tile_of(i) * kKeys + u;
         if (j < g.L_k) g.norm2[(int64_t)hk * g.L_k + j] = n2;  // pass 2 takes |k|^2 from here
         // rows past the end of the cache are zero-filled: 0 * (1 / 1e-12) = 0, they add nothing
@@ -380,19 +385,22 @@ score_tc_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constan
         for (int r = rg; r < kKeys; r += kGroups) {
           const uint4 w = lds_key_chunk<D>(tile, r, c);
           const float inv = sh->inv_s[vg][r];
+          const uint64_t inv2 = pack2(inv, inv);
           const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            acc[2 * e] = fmaf(fc::bf16_lo(ww[e]), inv, acc[2 * e]);
-            acc[2 * e + 1] = fmaf(fc::bf16_hi(ww[e]), inv, acc[2 * e + 1]);
-          }
+          for (int e = 0; e < 4; ++e) acc2[e] = fma2(pack2(fc::bf16_lo(ww[e]), fc::bf16_hi(ww[e])), inv2, acc2[e]);
         }
         named_barrier_128(1 + vg);  // inv_s[vg] is rewritten for this warpgroup's next tile
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sh->k_free[st]));
       }
 #pragma unroll
-      for (int e = 0; e < 8; ++e) sh->colsum_s[vg][rg][c * 8 + e] = acc[e];
+      for (int e = 0; e < 4; ++e) {
+        float lo, hi;
+        unpack2(acc2[e], lo, hi);
+        sh->colsum_s[vg][rg][c * 8 + 2 * e] = lo;
+        sh->colsum_s[vg][rg][c * 8 + 2 * e + 1] = hi;
+      }
       asm volatile("bar.sync 3, 256;" ::: "memory");  // both key-vector warpgroups
       if (vg == 0 && u < D) {
         float t = 0.f;
